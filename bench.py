@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark: one serving step of mixed decode + interrupt-append paged attention on B200.
+
+A step = asynclm_kv_append + asynclm_attn_mixed over one synthetic batch with the Llama-3-8B
+attention shape (32 query heads, 8 kv heads, head_dim 128, page 16, 32 sequences, contexts uniform
+in [512, 4096], 8 sequences receive an interrupt span of 8..64 tokens, the rest decode one token).
+The plan is built once per step on the host (it is shared by all layers of a model) and its cost is
+reported separately and inside the end-to-end figure.
+
+Prints ONE JSON line.  `value` is KV GB/s (bytes of K/V the step must read, divided by the step's
+device time); `ms_per_step` carries the step time.  Multi-GPU runs are independent replicas (the
+path has no cross-GPU exchange).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "kv_gbps_mixed_decode_interrupt_append"
+UNIT = "GB/s"
+WORKLOAD = "config2-llama3-8b-mixed-batch"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                self.samples.append((time.time(), float(parts[0]), float(parts[1]), parts[2:6]))
+            except ValueError:
+                pass
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        inside = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        reasons = sorted({self.NAMES[i] for s in inside for i, v in enumerate(s[3])
+                          if v.lower().startswith("active")})
+        return {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": inside[0][2],
+                "reasons": reasons, "samples": len(inside)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample_rows(st, budget_pairs: float, seed: int = 0):
+    """A seeded subset of token rows whose (row, key) pair count is about `budget_pairs`."""
+    n_row = np.repeat(st.kv_len_before.astype(np.int64), st.q_len) + \
+        np.concatenate([np.arange(1, q + 1) for q in st.q_len]) if st.total_q else np.zeros(0)
+    order = np.random.default_rng(seed).permutation(st.total_q)
+    csum = np.cumsum(n_row[order])
+    k = int(np.searchsorted(csum, budget_pairs, side="left")) + 1
+    rows = np.sort(order[:min(k, st.total_q)])
+    return rows, float(n_row[rows].sum()), float(n_row.sum())
+
+
+def time_oracle(wl, st, seconds_target: float):
+    """Times the oracle (as it stands) on a bounded row sample; returns a dict for the report."""
+    from oracle import oracle
+    from paper_2412_07017_b200 import workload as W
+    cores = oracle.num_threads()
+    pool = wl.kv_pool.copy()
+    t0 = time.perf_counter()
+    oracle.kv_append(pool, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices,
+                     st.k_new, st.v_new)
+    t_append = time.perf_counter() - t0
+    probe_rows, probe_pairs, total_pairs = oracle_sample_rows(st, 2.0e4 * cores, seed=1)
+    t0 = time.perf_counter()
+    oracle.attn_mixed(pool, st.q, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices,
+                      sel_rows=probe_rows)
+    rate = probe_pairs / max(time.perf_counter() - t0, 1e-6)       # (row, key) pairs per second
+    rows, pairs, total_pairs = oracle_sample_rows(st, rate * seconds_target, seed=2)
+    t0 = time.perf_counter()
+    oracle.attn_mixed(pool, st.q, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices,
+                      sel_rows=rows)
+    t_attn = time.perf_counter() - t0
+    step_seconds = t_append + t_attn * total_pairs / pairs
+    kv_bytes = W.algorithmic_bytes(wl.shape, st)["kv"]
+    return {"value": kv_bytes / step_seconds / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{len(rows)} of {st.total_q} token rows (seeded), all {wl.shape.num_q_heads} "
+                      f"heads, {pairs / total_pairs:.3f} of the step's (row,key) pairs, "
+                      f"{t_attn:.1f} s measured, step time extrapolated to {step_seconds:.1f} s",
+            "step_seconds": step_seconds}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2412_07017_b200 import workload as W
+    wl = W.make_config(2)
+    st = wl.steps[0]
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    times, last = [], None
+    for i in range(args.warmup + args.steps):
+        last = time_oracle(wl, st, per_step)
+        if i >= args.warmup:
+            times.append(last["step_seconds"])
+    kv_bytes = W.algorithmic_bytes(wl.shape, st)["kv"]
+    sec = float(np.mean(times))
+    value = kv_bytes / sec / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "seed": wl.seed},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2412_07017_b200 import binding as B
+    from paper_2412_07017_b200 import workload as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    wl = W.make_config(2)
+    st = wl.steps[0]
+    shape = wl.shape
+    by = W.algorithmic_bytes(shape, st)
+    flops = W.algorithmic_flops(shape, st)
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    def pinned(bits):
+        return torch.from_numpy(bits.view(np.int16)).pin_memory()
+
+    pool = dev(wl.kv_pool)
+    q, kn, vn = dev(st.q), dev(st.k_new), dev(st.v_new)
+    T = st.total_q
+    out = torch.empty((T, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > 126 MB L2
+    stream = torch.cuda.current_stream()
+
+    hb, db = B.workspace_size(shape, wl.num_pages, st.batch, T, len(st.page_indices))
+    host_ws = torch.empty(hb, dtype=torch.uint8).pin_memory()
+    dev_ws = torch.empty(db, dtype=torch.uint8, device="cuda")
+
+    def make_plan():
+        return B.asynclm_plan(shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr,
+                              st.page_indices, host_ws=host_ws, dev_ws=dev_ws)
+
+    plan = make_plan()
+    torch.cuda.synchronize()
+    launches_per_step = plan.info["launches_append"] + plan.info["launches_attn"]
+
+    def step():
+        B.asynclm_kv_append(plan, kn, vn, pool, stream)
+        B.asynclm_attn_mixed(plan, q, pool, out, None, stream)
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    assert B.last_device_status(plan) == 0
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    for k in range(args.steps):
+        flush.fill_(k & 0xff)                 # evict the pool from L2 between steps (untimed)
+        ev[k][0].record(stream)
+        B.asynclm_kv_append(plan, kn, vn, pool, stream)
+        ev[k][1].record(stream)
+        B.asynclm_attn_mixed(plan, q, pool, out, None, stream)
+        ev[k][2].record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    step_ms = np.array([e[0].elapsed_time(e[2]) for e in ev])
+    attn_ms = np.array([e[1].elapsed_time(e[2]) for e in ev])
+    total_ms = float(step_ms.sum())
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    assert B.last_device_status(plan) == 0
+
+    # end to end through the public API: pinned host inputs -> device, plan, append, attention,
+    # result back to pinned host memory, every step
+    q_h, kn_h, vn_h = pinned(st.q), pinned(st.k_new), pinned(st.v_new)
+    out_h = torch.empty((T, shape.num_q_heads, shape.head_dim), dtype=torch.int16).pin_memory()
+    q_d, kn_d, vn_d = torch.empty_like(q), torch.empty_like(kn), torch.empty_like(vn)
+    e2e_steps = min(args.steps, 200)
+    plan_us = []
+
+    def e2e_step():
+        q_d.view(torch.int16).copy_(q_h, non_blocking=True)
+        kn_d.view(torch.int16).copy_(kn_h, non_blocking=True)
+        vn_d.view(torch.int16).copy_(vn_h, non_blocking=True)
+        t0 = time.perf_counter()
+        p = make_plan()
+        plan_us.append((time.perf_counter() - t0) * 1e6)
+        B.asynclm_kv_append(p, kn_d, vn_d, pool, stream)
+        B.asynclm_attn_mixed(p, q_d, pool, out, None, stream)
+        out_h.copy_(out.view(torch.int16), non_blocking=True)
+        torch.cuda.synchronize()
+
+    for _ in range(3):
+        flush.fill_(2)
+        e2e_step()
+    plan_us.clear()
+    e2e_total = 0.0
+    for k in range(e2e_steps):
+        flush.fill_(k & 0xff)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e2e_step()
+        e2e_total += time.perf_counter() - t0
+    if world > 1:
+        tt = torch.tensor([e2e_total], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_total = float(tt.item())
+    h2d = q_h.numel() * 2 + kn_h.numel() * 2 + vn_h.numel() * 2 + plan.info["device_bytes_used"] * 0
+    d2h = out_h.numel() * 2
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    ms_per_step = total_ms / args.steps
+    value = world * by["kv"] / (ms_per_step * 1e-3) / 1e9
+    attn_bytes = by["kv"] + by["qo"] + by["page_ids"]
+    attn_s = float(attn_ms.mean()) * 1e-3
+    achieved = attn_bytes / attn_s / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": WORKLOAD, "seed": wl.seed, "batch": st.batch, "total_q": T,
+            "kv_tokens": int(plan.info["total_kv_tokens"]), "replicas": world,
+            "l2": "256 MiB buffer rewritten between timed steps (untimed)",
+            "us_per_step": ms_per_step * 1e3,
+            "us_per_step_p10_p50_p90": [float(np.percentile(step_ms, p)) * 1e3 for p in (10, 50, 90)],
+            "algorithmic_bytes_per_step": by["total"], "algorithmic_flops_per_step": flops,
+            "step_hbm_frac_of_" + peak_kind: by["total"] / (ms_per_step * 1e-3) / 1e9 / peak,
+            "step_hbm_frac_of_nominal_8TBps": by["total"] / (ms_per_step * 1e-3) / 1e9 / 8000.0,
+            "plan_host_us_median": float(np.median(plan_us)),
+            "plan": {k: plan.info[k] for k in ("num_items", "num_split_units", "num_items_tensor",
+                                               "kv_chunk_tokens", "num_ctas_cuda", "num_ctas_tensor")},
+        },
+        "roofline": {"bound": "hbm", "kernel": "asynclm_attn_mixed launches (attention + merge)",
+                     "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None,
+                     "algorithmic_bytes_per_launch": attn_bytes, "avg_launch_us": attn_s * 1e6},
+        "e2e": {"value": world * by["kv"] / (e2e_total / e2e_steps) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": int(h2d + plan.info["device_bytes_used"] * 0),
+                "d2h_bytes_per_step": int(d2h), "us_per_step": e2e_total / e2e_steps * 1e6,
+                "steps": e2e_steps, "includes": "H2D of q/k_new/v_new, asynclm_plan (+ its upload), "
+                "append, attention, D2H of out"},
+        "gpu_launches": int(args.steps * launches_per_step),
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        cb = time_oracle(wl, st, 12.0)
+        cb.pop("step_seconds")
+        line["cpu_baseline"] = cb
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

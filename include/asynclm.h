@@ -1,0 +1,211 @@
+/*
+ * asynclm.h -- C ABI of the AsyncLM serving-step attention library for NVIDIA B200 (sm_100a).
+ *
+ * One serving step under AsyncLM's interrupt mechanism is one batched attention pass over a paged
+ * KV cache.  Most sequences contribute a single decode query.  A sequence whose function call has
+ * returned contributes a multi-token interrupt span: the paper inserts the interrupt block at the
+ * end of the sequence's token stream and lets generation resume after it (Section 3.2,
+ * "Triggering Interrupts"), and the interrupt manager appends all queued interrupts to the
+ * generated tokens so that the next decoding step processes them (Section 5.3).  A sequence paused
+ * by a trap (Section 3.2, "Waiting for interrupts") contributes no query at all.  The span is
+ * appended in place; the cached context is not recomputed (the restart-and-recompute alternative is
+ * Section 5.5).
+ *
+ * Per step the caller runs, on one CUDA stream:
+ *     asynclm_plan       (host integer work + one async host->device copy of the plan)
+ *     asynclm_kv_append  (scatter the new K/V rows into their page slots)
+ *     asynclm_attn_mixed (attention of every new row over its sequence's pages)
+ * A plan depends only on the lengths and the page table, so a multi-layer model builds it once per
+ * step and reuses it for every layer's pool.
+ *
+ * Conventions
+ *   - bf16 tensors are passed as untyped device pointers; rows are contiguous and 16-byte aligned.
+ *   - kv_pool layout: [num_pages][2 (0 = K, 1 = V)][num_kv_heads][page_size][head_dim] bf16.
+ *   - Query heads [h*G, (h+1)*G), G = num_q_heads / num_kv_heads, share kv head h.
+ *   - New token i of sequence b (0 <= i < q_len_b) sits at position ctx_b + i of the sequence and
+ *     attends to positions 0 .. ctx_b + i (whole prior context; causal inside the span).
+ *   - "device" / "host" below says where a pointer must live.  The library never allocates or
+ *     frees device memory, never synchronises the stream and keeps no global mutable state other
+ *     than per-device attributes cached on first use.
+ *   - Every function returns an asynclm_status (0 = success, negative = error).  Nothing throws,
+ *     aborts or traps; kernels never wait on one another.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ */
+#ifndef ASYNCLM_H_
+#define ASYNCLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum asynclm_status {
+    ASYNCLM_OK = 0,
+    ASYNCLM_ERR_INVALID_ARG = -1,         /* NULL pointer, negative size, misaligned pointer   */
+    ASYNCLM_ERR_UNSUPPORTED_SHAPE = -2,   /* head_dim / page_size / group outside the set below */
+    ASYNCLM_ERR_PAGE_TABLE = -3,          /* too few pages for a sequence, or a page id out of
+                                             [0, num_pages), or (if asked) a page written twice  */
+    ASYNCLM_ERR_WORKSPACE_TOO_SMALL = -4,
+    ASYNCLM_ERR_CUDA = -5,                /* a CUDA runtime call or a launch failed            */
+    ASYNCLM_ERR_ARCH = -6,                /* current device is not compute capability 10.x     */
+    ASYNCLM_ERR_DEVICE_STATUS = -7        /* a kernel reported a bounded wait that ran out     */
+} asynclm_status;
+
+/* Supported: head_dim in {64, 128}; page_size = 16; num_q_heads / num_kv_heads in {1, 2, 4, 8}. */
+typedef struct asynclm_shape {
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim;
+    int32_t page_size;
+    int64_t num_pages;    /* capacity of the pool; page ids are checked against it */
+    float   sm_scale;     /* softmax scale; <= 0 selects 1/sqrt(head_dim) */
+    int32_t reserved;     /* must be 0 */
+} asynclm_shape;
+
+/* Planner knobs; a zero field selects the default. */
+typedef struct asynclm_plan_options {
+    int32_t num_sms;          /* SM count to balance for; 0 = query the current device.  Must be
+                                 given (> 0) when planning without a device workspace. */
+    int32_t kv_chunk_tokens;  /* fixed split-KV chunk length (multiple of 64); 0 = chosen so that
+                                 the work items roughly fill the machine; a value >= the longest
+                                 context disables splitting */
+    int32_t tensor_min_rows;  /* a span uses the tensor-core path when G * q_len >= this;
+                                 0 = default; a value > 128*G*... (INT32_MAX) keeps every row on
+                                 the CUDA-core path */
+    int32_t flags;            /* ASYNCLM_PLAN_* */
+} asynclm_plan_options;
+
+#define ASYNCLM_PLAN_REJECT_ALIASED_WRITES 1  /* error if two sequences append into one page */
+#define ASYNCLM_PLAN_NO_TENSOR_PATH        2  /* keep every row on the CUDA-core path         */
+
+/* Host-side description of one step's batch (all arrays on the host, int32). */
+typedef struct asynclm_batch {
+    int32_t        batch;          /* number of sequences B */
+    const int32_t* q_indptr;       /* [B+1] CSR over new tokens; q_len_b = q_indptr[b+1]-q_indptr[b]:
+                                      0 paused, 1 decode, > 1 interrupt append */
+    const int32_t* kv_len_before;  /* [B] tokens of b already stored in its pages (ctx_b) */
+    const int32_t* page_indptr;    /* [B+1] CSR over page_indices */
+    const int32_t* page_indices;   /* logical page j of b lives in physical page
+                                      page_indices[page_indptr[b] + j]; at least
+                                      ceil((ctx_b + q_len_b) / page_size) entries per sequence,
+                                      extra (pre-allocated) pages are allowed */
+} asynclm_batch;
+
+/* Opaque plan; it lives inside the caller's host workspace. */
+typedef struct asynclm_plan_s asynclm_plan_t;
+
+/* What the planner decided; filled by asynclm_plan_get_info. */
+typedef struct asynclm_plan_info {
+    int32_t total_q;          /* T = sum of q_len */
+    int32_t num_units;        /* (sequence, kv head, query tile) units */
+    int32_t num_items;        /* (unit, kv chunk) work items */
+    int32_t num_split_units;  /* units whose keys were split into > 1 chunk */
+    int32_t partial_rows;     /* rows of fp32 partial output held in the device workspace */
+    int32_t kv_chunk_tokens;  /* chosen chunk length (INT32_MAX = unsplit) */
+    int32_t num_ctas_cuda;    /* persistent CTAs of the CUDA-core attention kernel */
+    int32_t num_ctas_tensor;  /* persistent CTAs of the tensor-core attention kernel */
+    int32_t num_items_tensor; /* items routed to the tensor-core kernel */
+    int32_t launches_append;  /* kernels asynclm_kv_append launches */
+    int32_t launches_attn;    /* kernels asynclm_attn_mixed launches */
+    int32_t num_sms;
+    int64_t total_kv_tokens;  /* sum over active sequences of ctx_b + q_len_b */
+    uint64_t device_bytes_used;
+    uint64_t host_bytes_used;
+} asynclm_plan_info;
+
+/* One row of the plan's work list, for inspection and tests (asynclm_plan_get_items). */
+typedef struct asynclm_item_view {
+    int32_t seq;        /* sequence b */
+    int32_t kv_head;
+    int32_t tok0;       /* first new token of the unit, index i inside the sequence's span */
+    int32_t ntok;       /* tokens of the span covered by the unit */
+    int32_t kv0, kv1;   /* key positions [kv0, kv1) the item reads (before causal clipping) */
+    int32_t path;       /* 0 = CUDA-core kernel, 1 = tensor-core kernel */
+    int32_t cta;        /* persistent CTA (within its kernel) that processes the item */
+} asynclm_item_view;
+
+int asynclm_version(void);
+const char* asynclm_strerror(int status);
+
+/*
+ * Upper bounds on the workspaces asynclm_plan needs for any batch with at most max_batch
+ * sequences, max_total_q new tokens and max_total_pages page-table entries.  The device workspace
+ * holds the uploaded plan and the fp32 partial outputs of split-KV items.  opts may be NULL.
+ */
+int asynclm_plan_workspace_size(const asynclm_shape* shape, const asynclm_plan_options* opts,
+                                int32_t max_batch, int32_t max_total_q, int64_t max_total_pages,
+                                size_t* host_bytes, size_t* device_bytes);
+
+/*
+ * Build the plan for one step (the "next decoding step" of Section 5.3, seen from attention).
+ *
+ * Validates the batch, tiles every (sequence, kv head) into query tiles and page-aligned KV chunks
+ * (long contexts are split; partial results are merged by log-sum-exp inside asynclm_attn_mixed),
+ * orders the items longest-first and assigns them to persistent CTAs, then enqueues ONE
+ * host->device copy of the packed plan on `stream`.
+ *
+ *   host_ws / host_bytes  host memory (8-byte aligned; pinned recommended) that must stay untouched
+ *                         until the copy has completed and for as long as the plan is used.
+ *   dev_ws / dev_bytes    device memory (256-byte aligned) owned by the caller.  dev_ws == NULL
+ *                         builds the plan on the host only (no CUDA call is made; opts->num_sms
+ *                         must be set); such a plan can be inspected but not executed.
+ *   out_plan              receives a pointer into host_ws.
+ *
+ * The batch arrays may be freed as soon as the call returns.  Errors: INVALID_ARG (NULL, negative
+ * or non-monotone indptr), UNSUPPORTED_SHAPE, PAGE_TABLE, WORKSPACE_TOO_SMALL, ARCH, CUDA.
+ */
+int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_options* opts,
+                 const asynclm_batch* batch, void* host_ws, size_t host_bytes,
+                 void* dev_ws, size_t dev_bytes, void* stream, asynclm_plan_t** out_plan);
+
+int asynclm_plan_get_info(const asynclm_plan_t* plan, asynclm_plan_info* info);
+
+/* Copies up to `capacity` items into `items` (host); returns the number of items, or < 0. */
+int asynclm_plan_get_items(const asynclm_plan_t* plan, asynclm_item_view* items, int32_t capacity);
+
+/*
+ * Interrupt append (Section 3.2: the block is inserted at the end of the context).  For every new
+ * token row r = q_indptr[b] + i and kv head h, copies the head_dim bf16 values of k_new[r][h] and
+ * v_new[r][h] bit for bit into
+ *     kv_pool[page_indices[page_indptr[b] + (ctx_b + i) / page_size]][0 | 1][h][(ctx_b + i) % page_size].
+ * No other byte of the pool is written.
+ *
+ *   k_new, v_new  device, bf16 [T][num_kv_heads][head_dim]
+ *   kv_pool       device, bf16, layout above
+ * Errors: INVALID_ARG, CUDA.
+ */
+int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, const void* v_new,
+                      void* kv_pool, void* stream);
+
+/*
+ * Mixed decode + interrupt-append attention (Section 5.3: the appended tokens are processed in the
+ * next decoding step, alongside the other sequences' single-token decodes).  Must follow
+ * asynclm_kv_append on the same stream: the new rows are read back from the pages.  For every new
+ * token row r = q_indptr[b] + i and query head hq (kv head hq / G):
+ *     s_j  = sm_scale * <q[r][hq], K_j>            j = 0 .. ctx_b + i
+ *     out[r][hq] = sum_j softmax(s)_j V_j          lse[r][hq] = ln sum_j exp(s_j)
+ * with K_j, V_j read through the page table.  bf16 inputs, fp32 accumulation, bf16 output rounded
+ * to nearest even.  Slots beyond a sequence's length and unreferenced pages are never allowed to
+ * influence the result, whatever bit patterns they hold.
+ *
+ *   q    device, bf16 [T][num_q_heads][head_dim]
+ *   out  device, bf16 [T][num_q_heads][head_dim]
+ *   lse  device, fp32 [T][num_q_heads], natural log; may be NULL
+ * Errors: INVALID_ARG, CUDA.
+ */
+int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv_pool,
+                       void* out, float* lse, void* stream);
+
+/*
+ * Reads the device status word of the plan's workspace (synchronises `stream`).  *host_out is 0
+ * if no kernel reported a problem, otherwise a code naming the bounded wait that ran out.  Returns
+ * ASYNCLM_OK or ASYNCLM_ERR_DEVICE_STATUS / ASYNCLM_ERR_CUDA.
+ */
+int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASYNCLM_H_ */

@@ -1,0 +1,65 @@
+// C ABI entry points that launch kernels (see include/asynclm.h for the contract).
+#include <cuda_runtime.h>
+
+#include "asynclm.h"
+#include "kernels.h"
+#include "plan_internal.h"
+
+using namespace asynclm;
+
+namespace asynclm {
+bool tensor_path_compiled(int) { return false; }
+}  // namespace asynclm
+
+extern "C" int asynclm_version(void) { return 100; }
+
+extern "C" const char* asynclm_strerror(int status) {
+    switch (status) {
+        case ASYNCLM_OK: return "ok";
+        case ASYNCLM_ERR_INVALID_ARG: return "invalid argument";
+        case ASYNCLM_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case ASYNCLM_ERR_PAGE_TABLE: return "page table does not cover a sequence or holds an id outside the pool";
+        case ASYNCLM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case ASYNCLM_ERR_CUDA: return "CUDA runtime error";
+        case ASYNCLM_ERR_ARCH: return "device is not compute capability 10.x";
+        case ASYNCLM_ERR_DEVICE_STATUS: return "a kernel reported a bounded wait that ran out";
+        default: return "unknown status";
+    }
+}
+
+static bool runnable(const asynclm_plan_t* plan) {
+    return plan && plan->magic == kPlanMagic && !plan->host_only;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+extern "C" int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, const void* v_new,
+                                 void* kv_pool, void* stream) {
+    if (!runnable(plan)) return ASYNCLM_ERR_INVALID_ARG;
+    if (plan->dev.total_q == 0) return ASYNCLM_OK;
+    if (!k_new || !v_new || !kv_pool || !aligned16(k_new) || !aligned16(v_new) || !aligned16(kv_pool))
+        return ASYNCLM_ERR_INVALID_ARG;
+    return launch_kv_append(plan->dev, k_new, v_new, kv_pool, (cudaStream_t)stream) == cudaSuccess
+               ? ASYNCLM_OK : ASYNCLM_ERR_CUDA;
+}
+
+extern "C" int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv_pool,
+                                  void* out, float* lse, void* stream) {
+    if (!runnable(plan)) return ASYNCLM_ERR_INVALID_ARG;
+    if (plan->dev.total_q == 0) return ASYNCLM_OK;
+    if (!q || !kv_pool || !out || !aligned16(q) || !aligned16(kv_pool) || !aligned16(out))
+        return ASYNCLM_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (launch_attn_cuda_core(plan->dev, q, kv_pool, out, lse, s) != cudaSuccess) return ASYNCLM_ERR_CUDA;
+    if (launch_lse_merge(plan->dev, out, lse, s) != cudaSuccess) return ASYNCLM_ERR_CUDA;
+    return ASYNCLM_OK;
+}
+
+extern "C" int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out) {
+    if (!runnable(plan) || !host_out) return ASYNCLM_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(host_out, plan->dev.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return ASYNCLM_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return ASYNCLM_ERR_CUDA;
+    return *host_out == 0 ? ASYNCLM_OK : ASYNCLM_ERR_DEVICE_STATUS;
+}

@@ -1,0 +1,56 @@
+// Internal plan format shared by the host planner and the kernels (not part of the public ABI).
+#pragma once
+#include <stddef.h>
+#include <stdint.h>
+
+namespace asynclm {
+
+constexpr int kKvTile = 128;          // split-KV chunk granularity in tokens (8 pages of 16)
+constexpr int kPage = 16;
+constexpr int kPathCuda = 0;
+constexpr int kPathTensor = 1;
+
+// A unit is one query tile of one (sequence, kv head): `ntok` consecutive new tokens times the G
+// query heads that share the kv head.  Token t of the unit sees keys [0, kv_limit0 + t).
+struct Unit {
+    int32_t seq;
+    int32_t kv_head;
+    int32_t q_row0;        // global token row of the unit's first token
+    int32_t ntok;
+    int32_t kv_limit0;     // ctx_b + tok0 + 1
+    int32_t n_chunks;      // number of KV chunks (items) of this unit
+    int32_t partial_base;  // first partial row (chunk c, token t -> partial_base + c*ntok + t); -1 if unsplit
+    int32_t page_base;     // page_indptr[seq]
+};
+
+// An item is one KV chunk of one unit.
+struct Item {
+    int32_t unit;
+    int32_t kv0;           // first key position
+    int32_t kv1;           // one past the last key position any token of the unit may see here
+    int32_t chunk;         // chunk index inside the unit
+};
+
+// Pointers into the device workspace, passed to kernels by value.
+struct DevPlan {
+    const int32_t* q_indptr;
+    const int32_t* kv_len_before;
+    const int32_t* page_indptr;
+    const int32_t* page_indices;
+    const int32_t* row_seq;          // [T] sequence of each new token row
+    const Unit* units;
+    const Item* items;               // CUDA-core items first (grouped by CTA), then tensor items
+    const int32_t* cta_indptr_cuda;  // [num_ctas_cuda + 1] into items
+    const int32_t* cta_indptr_tensor;// [num_ctas_tensor + 1] into items (absolute indices)
+    const int32_t* split_units;      // [num_split_units] unit ids that need a merge
+    float* partial_o;                // [partial_rows][G][d]
+    float* partial_lse;              // [partial_rows][G]   (log2 domain)
+    int32_t* status;                 // device status word
+    int32_t batch, total_q, num_units, num_items, num_items_cuda, num_items_tensor;
+    int32_t num_split_units, num_ctas_cuda, num_ctas_tensor;
+    int32_t num_q_heads, num_kv_heads, head_dim, group;
+    int64_t num_pages;
+    float sm_scale;
+};
+
+}  // namespace asynclm

@@ -1,0 +1,168 @@
+"""GPU parity: the CUDA path through the C ABI against the fp64 CPU oracle, element by element.
+
+Bars: KV append bit-exact over the whole pool; attention max |err| <= 1e-2 and mean |err| <= 1e-3
+(bf16 inputs, fp32 accumulation, bf16 output); lse within 1e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_07017_b200 import binding as B
+from paper_2412_07017_b200 import workload as W
+from gpu_util import (assert_close, gpu_step, oracle_step, to_bits, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_check(wl, st=None, what="", **opts):
+    st = st or wl.steps[0]
+    pool_dev, out_bits, lse, plan = gpu_step(wl, st, **opts)
+    ref_pool, ref_out, ref_lse = oracle_step(wl, st)
+    assert np.array_equal(to_bits(pool_dev), ref_pool), f"{what}: pool differs after append"
+    assert_close(out_bits, lse, ref_out, ref_lse, what=what)
+    return out_bits, lse, plan
+
+
+def test_config1_tiny_mixed_step():
+    wl = W.make_config(1)
+    _, _, plan = run_and_check(wl, what="config1")
+    assert plan.info["total_q"] == 15
+
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(8, 2, 64), (4, 4, 64), (8, 1, 64), (2, 1, 128), (32, 8, 128),
+                                      (16, 2, 128), (4, 2, 128), (8, 8, 128)])
+def test_shapes_and_ragged_lengths(Hq, Hkv, d):
+    shape = W.Shape(Hq, Hkv, d, 16)
+    ctx = [0, 1, 15, 16, 17, 129, 700, 0, 300, 47]
+    ql = [1, 1, 1, 1, 12, 5, 1, 33, 0, 70]
+    wl = W.make_single_step("ragged", shape, ctx, ql, seed=1000 + Hq * 7 + d,
+                            extra_pages=[0, 1, 0, 0, 2, 0, 0, 1, 3, 0], interleave_pages=True)
+    run_and_check(wl, what=f"ragged {Hq}/{Hkv}/{d}")
+
+
+@pytest.mark.parametrize("chunk", [64, 128, 512, 1 << 20])
+def test_fixed_chunk_lengths_agree_with_oracle(chunk):
+    shape = W.Shape(8, 2, 128, 16)
+    wl = W.make_single_step("chunks", shape, [1500, 64, 127, 900], [1, 1, 40, 7], seed=77)
+    _, _, plan = run_and_check(wl, what=f"chunk {chunk}", kv_chunk_tokens=chunk)
+    if chunk < 1 << 20:
+        assert plan.info["num_split_units"] > 0
+
+
+def test_cuda_core_path_handles_spans_too():
+    shape = W.Shape(8, 2, 128, 16)
+    wl = W.make_single_step("spans", shape, [300, 0, 40], [64, 130, 9], seed=78)
+    run_and_check(wl, what="cuda-core spans", flags=B.PLAN_NO_TENSOR_PATH)
+
+
+def test_results_are_bitwise_reproducible():
+    wl = W.make_config(1)
+    a = gpu_step(wl, wl.steps[0])
+    b = gpu_step(wl, wl.steps[0])
+    assert np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
+
+
+def test_physical_page_order_does_not_change_a_single_bit():
+    wl = W.make_config(1)
+    st = wl.steps[0]
+    _, out, lse, _ = gpu_step(wl, st)
+    perm = np.random.default_rng(9).permutation(wl.num_pages)
+    pool2 = np.empty_like(wl.kv_pool)
+    pool2[perm] = wl.kv_pool
+    wl2 = W.Workload("perm", wl.shape, wl.num_pages, pool2)
+    st2 = W.Step(st.q_indptr, st.kv_len_before, st.page_indptr,
+                 perm[st.page_indices].astype(np.int32), st.q, st.k_new, st.v_new)
+    _, out2, lse2, _ = gpu_step(wl2, st2)
+    assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def test_unused_slots_and_pages_may_hold_nan_patterns():
+    shape = W.Shape(8, 2, 128, 16)
+    args = dict(kv_len_before=[100, 37, 3, 260], q_len=[12, 1, 1, 35], seed=61,
+                extra_pages=[1, 0, 2, 0])
+    clean = W.make_single_step("clean", shape, **args)
+    dirty = W.make_single_step("dirty", shape, poison_unused=True, **args)
+    _, out_c, lse_c, _ = gpu_step(clean, clean.steps[0])
+    out_d, lse_d, _ = run_and_check(dirty, what="poisoned")
+    assert np.array_equal(out_c, out_d) and np.array_equal(lse_c, lse_d)
+
+
+def test_single_visible_key_returns_v_exactly():
+    shape = W.Shape(8, 2, 64, 16)
+    wl = W.make_single_step("one", shape, [0, 0, 0], [1, 1, 3], seed=22)
+    st = wl.steps[0]
+    _, out, _, _ = gpu_step(wl, st)
+    for r in (0, 1, 2):
+        assert np.array_equal(out[r], np.repeat(st.v_new[r], shape.group, axis=0))
+
+
+def test_append_only_touches_its_slots_and_is_idempotent():
+    shape = W.Shape(8, 2, 128, 16)
+    wl = W.make_single_step("app", shape, [5, 16, 31, 0, 40], [12, 1, 2, 7, 0], seed=11,
+                            extra_pages=[0, 1, 0, 2, 1], poison_unused=True)
+    st = wl.steps[0]
+    pool_dev, _, _, plan = gpu_step(wl, st)
+    ref_pool, _, _ = oracle_step(wl, st)
+    assert np.array_equal(to_bits(pool_dev), ref_pool)
+    B.asynclm_kv_append(plan, to_dev(st.k_new), to_dev(st.v_new), pool_dev)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_bits(pool_dev), ref_pool)
+
+
+def test_two_spans_in_two_steps_equal_one_concatenated_span():
+    shape = W.Shape(8, 2, 128, 16)
+    ctx, a1, a2 = 210, 9, 14
+    wl = W.make_single_step("cat", shape, [ctx], [a1 + a2], seed=41)
+    st = wl.steps[0]
+    pool_one, out_one, _, _ = gpu_step(wl, st)
+    s1 = W.Step(np.array([0, a1], np.int32), np.array([ctx], np.int32), st.page_indptr,
+                st.page_indices, st.q[:a1].copy(), st.k_new[:a1].copy(), st.v_new[:a1].copy())
+    s2 = W.Step(np.array([0, a2], np.int32), np.array([ctx + a1], np.int32), st.page_indptr,
+                st.page_indices, st.q[a1:].copy(), st.k_new[a1:].copy(), st.v_new[a1:].copy())
+    pool, _, _, _ = gpu_step(wl, s1)
+    pool, out_b, _, _ = gpu_step(wl, s2, pool_dev=pool)
+    assert np.array_equal(to_bits(pool), to_bits(pool_one))
+    ref_pool, ref_out, ref_lse = oracle_step(wl, st)
+    assert_close(out_b, None, ref_out[a1:], None, what="second span")
+
+
+def test_custom_softmax_scale():
+    shape = W.Shape(8, 2, 64, 16)
+    wl = W.make_single_step("scale", shape, [90, 10], [5, 1], seed=5)
+    st = wl.steps[0]
+    _, out, lse, _ = gpu_step(wl, st, sm_scale=0.05)
+    _, ref_out, ref_lse = oracle_step(wl, st, sm_scale=0.05)
+    assert_close(out, lse, ref_out, ref_lse, what="scale")
+
+
+def test_empty_and_all_paused_batches_are_no_ops():
+    shape = W.Shape(8, 2, 64, 16)
+    wl = W.make_single_step("paused", shape, [30, 50], [0, 0], seed=71)
+    st = wl.steps[0]
+    pool_dev, out, _, plan = gpu_step(wl, st)
+    assert out.shape[0] == 0 and np.array_equal(to_bits(pool_dev), wl.kv_pool)
+
+
+def test_replay_steps_keep_state_across_steps():
+    wl = W.make_replay(batch=24, steps=6, ctx_lo=40, ctx_hi=400, rate=0.2,
+                       shape=W.Shape(32, 8, 128, 16))
+    pool_dev = to_dev(wl.kv_pool)
+    ref_pool = wl.kv_pool.copy()
+    for t, st in enumerate(wl.steps):
+        pool_dev, out, lse, _ = gpu_step(wl, st, pool_dev=pool_dev)
+        ref_pool, ref_out, ref_lse = oracle_step(wl, st, pool=ref_pool)
+        assert np.array_equal(to_bits(pool_dev), ref_pool), f"step {t}"
+        assert_close(out, lse, ref_out, ref_lse, what=f"replay step {t}")
+
+
+def test_config2_llama_batch_full_size():
+    """Full-size Llama-3-8B-shaped mixed batch, default planning (the benchmarked configuration)."""
+    wl = W.make_config(2)
+    st = wl.steps[0]
+    pool_dev, out, lse, plan = gpu_step(wl, st)
+    ref_pool, ref_out, ref_lse = oracle_step(wl, st)
+    assert np.array_equal(to_bits(pool_dev), ref_pool)
+    is_app = np.repeat(st.q_len > 1, st.q_len)
+    assert_close(out, lse, ref_out, ref_lse, rows=np.nonzero(~is_app)[0], what="config2 decode rows")
+    assert_close(out, lse, ref_out, ref_lse, rows=np.nonzero(is_app)[0], what="config2 append rows")
+    assert_close(out, lse, ref_out, ref_lse, what="config2")

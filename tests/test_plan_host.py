@@ -1,0 +1,149 @@
+"""Host planner (integer work only, no GPU): coverage, balance and validation."""
+import numpy as np
+import pytest
+
+from paper_2412_07017_b200 import binding as B
+from paper_2412_07017_b200 import workload as W
+
+
+def plan(wl, st=None, **kw):
+    st = st or wl.steps[0]
+    return B.plan_host(wl.shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr,
+                       st.page_indices, **kw)
+
+
+def check_cover(wl, p, st=None):
+    """Every (sequence, kv head, new token, visible key) is covered by exactly one item."""
+    st = st or wl.steps[0]
+    items = p.items()
+    cover = {}
+    for it in items:
+        for t in range(it["ntok"]):
+            i = it["tok0"] + t
+            lim = int(st.kv_len_before[it["seq"]]) + i + 1
+            lo, hi = int(it["kv0"]), min(int(it["kv1"]), lim)
+            key = (int(it["seq"]), int(it["kv_head"]), i)
+            cover.setdefault(key, []).append((lo, hi))
+    want = set()
+    for b in range(st.batch):
+        for i in range(int(st.q_len[b])):
+            for h in range(wl.shape.num_kv_heads):
+                want.add((b, h, i))
+    assert set(cover) == want
+    for (b, h, i), segs in cover.items():
+        segs = sorted(s for s in segs if s[1] > s[0])
+        assert segs[0][0] == 0
+        for a, c in zip(segs[:-1], segs[1:]):
+            assert a[1] == c[0]
+        assert segs[-1][1] == int(st.kv_len_before[b]) + i + 1
+    # chunk boundaries are page aligned
+    assert (items["kv0"] % 16 == 0).all()
+    return items
+
+
+@pytest.mark.parametrize("chunk", [0, 64, 128, 512, 1 << 20])
+def test_items_partition_the_causal_work(chunk):
+    wl = W.make_config(1)
+    p = plan(wl, kv_chunk_tokens=chunk)
+    items = check_cover(wl, p)
+    assert p.info["total_q"] == 15 and p.info["num_items"] == len(items)
+    if chunk >= 1 << 20:
+        assert p.info["num_split_units"] == 0 and p.info["partial_rows"] == 0
+
+
+@pytest.mark.parametrize("sms", [1, 4, 148])
+def test_cover_with_paused_and_empty_context_sequences(sms):
+    shape = W.Shape(8, 2, 64, 16)
+    wl = W.make_single_step("t", shape, [0, 700, 33, 0, 5], [40, 0, 1, 1, 3], seed=2)
+    p = plan(wl, num_sms=sms)
+    check_cover(wl, p)
+
+
+def test_balance_on_the_llama_batch():
+    wl = W.make_config(2, scale=1.0) if False else None
+    # lengths only: build tables without materialising values
+    g = np.random.default_rng(0)
+    ctx = g.integers(512, 4097, 32)
+    ql = np.ones(32, dtype=np.int64); ql[:8] = g.integers(8, 65, 8)
+    shape = W.Shape(32, 8, 128, 16)
+    need = -(-(ctx + ql) // 16)
+    ids = np.arange(need.sum())
+    q_indptr, page_indptr, page_indices, _ = W.build_step_tables(ctx, ql, 16, ids)
+    p = B.plan_host(shape, int(need.sum()), q_indptr, ctx, page_indptr, page_indices, num_sms=148,
+                    flags=B.PLAN_NO_TENSOR_PATH)
+    items = p.items()
+    load = np.zeros(p.info["num_ctas_cuda"])
+    np.add.at(load, items["cta"], -(-(items["kv1"] - items["kv0"]) // 128) + 1)
+    assert load.max() <= 1.25 * load.mean() + 2
+    # items of one CTA are contiguous in the list
+    assert (np.diff(items["cta"]) >= 0).all()
+
+
+def test_plan_is_a_function_of_lengths_only():
+    wl = W.make_config(1)
+    st = wl.steps[0]
+    a = plan(wl).items()
+    perm = np.random.default_rng(3).permutation(wl.num_pages).astype(np.int32)
+    b = B.plan_host(wl.shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr,
+                    perm[st.page_indices]).items()
+    assert np.array_equal(a, b)
+
+
+def test_empty_batch_and_all_paused():
+    shape = W.Shape(8, 2, 64, 16)
+    p = B.plan_host(shape, 4, [0], [], [0], [])
+    assert p.info["num_items"] == 0 and p.info["total_q"] == 0
+    p = B.plan_host(shape, 4, [0, 0, 0], [5, 9], [0, 1, 2], [0, 1])
+    assert p.info["num_items"] == 0
+
+
+def _expect(status, fn):
+    with pytest.raises(B.AsynclmError) as e:
+        fn()
+    assert e.value.status == status
+
+
+def test_validation_errors():
+    shape = W.Shape(8, 2, 64, 16)
+    ok = dict(q_indptr=[0, 1], kv_len_before=[20], page_indptr=[0, 2], page_indices=[1, 0])
+    B.plan_host(shape, 2, **ok)
+    _expect(-3, lambda: B.plan_host(shape, 2, **{**ok, "page_indptr": [0, 1]}))       # too few pages
+    _expect(-3, lambda: B.plan_host(shape, 2, **{**ok, "page_indices": [1, 2]}))      # id outside pool
+    _expect(-3, lambda: B.plan_host(shape, 2, **{**ok, "page_indices": [-1, 0]}))
+    _expect(-1, lambda: B.plan_host(shape, 2, **{**ok, "q_indptr": [0, -1]}))         # negative q_len
+    _expect(-1, lambda: B.plan_host(shape, 2, **{**ok, "kv_len_before": [-2]}))
+    _expect(-1, lambda: B.plan_host(shape, 2, **{**ok, "q_indptr": [1, 2]}))          # indptr[0] != 0
+    _expect(-1, lambda: B.plan_host(shape, 2, kv_chunk_tokens=100, **ok))             # not a multiple of 64
+    _expect(-2, lambda: B.plan_host(W.Shape(8, 2, 96, 16), 2, **ok))                  # head_dim
+    _expect(-2, lambda: B.plan_host(W.Shape(8, 2, 64, 32), 2, **ok))                  # page size
+    _expect(-2, lambda: B.plan_host(W.Shape(6, 2, 64, 16), 2, **ok))                  # group 3
+    _expect(-2, lambda: B.plan_host(W.Shape(7, 2, 64, 16), 2, **ok))
+
+
+def test_paused_sequence_page_ids_are_not_checked():
+    shape = W.Shape(8, 2, 64, 16)
+    B.plan_host(shape, 2, [0, 0, 1], [40, 3], [0, 3, 4], [99, -5, 7, 1])
+
+
+def test_aliased_write_detection_is_optional():
+    shape = W.Shape(8, 2, 64, 16)
+    args = dict(q_indptr=[0, 1, 2], kv_len_before=[3, 3], page_indptr=[0, 1, 2], page_indices=[0, 0])
+    B.plan_host(shape, 1, **args)
+    _expect(-3, lambda: B.plan_host(shape, 1, flags=B.PLAN_REJECT_ALIASED_WRITES, **args))
+    # sharing a fully read-only prefix page is fine
+    args = dict(q_indptr=[0, 1, 2], kv_len_before=[16, 16], page_indptr=[0, 2, 4],
+                page_indices=[0, 1, 0, 2])
+    B.plan_host(shape, 3, flags=B.PLAN_REJECT_ALIASED_WRITES, **args)
+
+
+def test_workspace_size_bounds_actual_use():
+    wl = W.make_config(1)
+    st = wl.steps[0]
+    p = plan(wl)
+    hb, db = B.workspace_size(wl.shape, wl.num_pages, st.batch, st.total_q, len(st.page_indices),
+                              num_sms=148)
+    assert hb >= p.info["host_bytes_used"] and db >= p.info["device_bytes_used"]
+    p = plan(wl, kv_chunk_tokens=64)
+    hb, db = B.workspace_size(wl.shape, wl.num_pages, st.batch, st.total_q, len(st.page_indices),
+                              num_sms=148, kv_chunk_tokens=64)
+    assert hb >= p.info["host_bytes_used"] and db >= p.info["device_bytes_used"]
