@@ -128,6 +128,9 @@ typedef struct asynclm_item_view {
 
 int asynclm_version(void);
 const char* asynclm_strerror(int status);
+/* Text of the CUDA error behind the calling thread's most recent ASYNCLM_ERR_CUDA from
+   asynclm_kv_append / asynclm_attn_mixed ("no error" if there was none). */
+const char* asynclm_last_cuda_error(void);
 
 /*
  * Upper bounds on the workspaces asynclm_plan needs for any batch with at most max_batch

@@ -19,7 +19,7 @@ from . import build as _build
 EXPORTS = [
     "asynclm_version", "asynclm_strerror", "asynclm_plan_workspace_size", "asynclm_plan",
     "asynclm_plan_get_info", "asynclm_plan_get_items", "asynclm_kv_append", "asynclm_attn_mixed",
-    "asynclm_last_device_status",
+    "asynclm_last_device_status", "asynclm_last_cuda_error",
 ]
 
 PLAN_REJECT_ALIASED_WRITES = 1
@@ -29,7 +29,8 @@ PLAN_NO_TENSOR_PATH = 2
 class AsynclmError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
-        super().__init__(f"{what}: {strerror(status)} ({status})")
+        detail = f" [{load().asynclm_last_cuda_error().decode()}]" if status == -5 else ""
+        super().__init__(f"{what}: {strerror(status)} ({status}){detail}")
 
 
 class CShape(ctypes.Structure):
@@ -85,6 +86,7 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_version.restype = ctypes.c_int
     lib.asynclm_strerror.restype = ctypes.c_char_p
     lib.asynclm_strerror.argtypes = [ctypes.c_int]
+    lib.asynclm_last_cuda_error.restype = ctypes.c_char_p
     lib.asynclm_plan_workspace_size.argtypes = [ctypes.POINTER(CShape), ctypes.POINTER(CPlanOptions),
                                                 i32, i32, i64, szp, szp]
     lib.asynclm_plan.argtypes = [ctypes.POINTER(CShape), ctypes.POINTER(CPlanOptions),
@@ -96,7 +98,7 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_attn_mixed.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.asynclm_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     for name in EXPORTS:
-        if name != "asynclm_strerror":
+        if name not in ("asynclm_strerror", "asynclm_last_cuda_error"):
             getattr(lib, name).restype = ctypes.c_int
     _lib = lib
     return lib

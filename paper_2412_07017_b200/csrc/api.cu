@@ -11,7 +11,18 @@ namespace asynclm {
 bool tensor_path_compiled(int) { return false; }
 }  // namespace asynclm
 
+static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+static int cuda_status(cudaError_t e) {
+    if (e == cudaSuccess) return ASYNCLM_OK;
+    g_last_cuda_error = e;
+    (void)cudaGetLastError();   // clear the sticky launch-configuration error, if that is what it was
+    return ASYNCLM_ERR_CUDA;
+}
+
 extern "C" int asynclm_version(void) { return 100; }
+
+extern "C" const char* asynclm_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 extern "C" const char* asynclm_strerror(int status) {
     switch (status) {
@@ -39,8 +50,7 @@ extern "C" int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, 
     if (plan->dev.total_q == 0) return ASYNCLM_OK;
     if (!k_new || !v_new || !kv_pool || !aligned16(k_new) || !aligned16(v_new) || !aligned16(kv_pool))
         return ASYNCLM_ERR_INVALID_ARG;
-    return launch_kv_append(plan->dev, k_new, v_new, kv_pool, (cudaStream_t)stream) == cudaSuccess
-               ? ASYNCLM_OK : ASYNCLM_ERR_CUDA;
+    return cuda_status(launch_kv_append(plan->dev, k_new, v_new, kv_pool, (cudaStream_t)stream));
 }
 
 extern "C" int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv_pool,
@@ -50,9 +60,9 @@ extern "C" int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, con
     if (!q || !kv_pool || !out || !aligned16(q) || !aligned16(kv_pool) || !aligned16(out))
         return ASYNCLM_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
-    if (launch_attn_cuda_core(plan->dev, q, kv_pool, out, lse, s) != cudaSuccess) return ASYNCLM_ERR_CUDA;
-    if (launch_lse_merge(plan->dev, out, lse, s) != cudaSuccess) return ASYNCLM_ERR_CUDA;
-    return ASYNCLM_OK;
+    int rc = cuda_status(launch_attn_decode(plan->dev, q, kv_pool, out, lse, s));
+    if (rc != ASYNCLM_OK) return rc;
+    return cuda_status(launch_lse_merge(plan->dev, out, lse, s));
 }
 
 extern "C" int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out) {

@@ -1,0 +1,485 @@
+// CUDA-core attention for decode rows (and spans too short for the tensor-core path).
+//
+// Each new token attends to its sequence's whole cached context plus its own span up to itself
+// (paper Section 3.2 / 5.3: interrupt tokens are appended to the context and processed in the next
+// decoding step, next to the other sequences' one-token decodes).  This path is bound by HBM
+// bandwidth: every K/V row is read once and used by the G query heads that share the kv head.
+//
+// Structure: one persistent CTA per SM walks the item list the planner gave it.  A producer warp
+// streams the items' K/V pages (contiguous 16-token blocks) into a shared-memory ring with bulk
+// asynchronous copies that complete on mbarriers, together with a small descriptor and the query
+// rows of each item.  Eight consumer warps each take 8 of a tile's 64 rows: fp32 dot products with
+// packed two-wide FMAs, a transposing shuffle reduction, softmax against a lazily updated reference
+// maximum, and the P.V update; at the end of an item the warps' states are merged through shared
+// memory and written either as final bf16 output or as an fp32 partial for the split-KV merge.
+//
+// Every wait is bounded: a wait that runs out sets the plan's device status word and a CTA-wide
+// abort flag, after which all loops fall through and the kernel returns.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace asynclm {
+
+namespace dec {
+
+constexpr int kWarps = 8;                    // consumer warps
+constexpr int kThreads = (kWarps + 1) * 32;  // + 1 producer warp
+constexpr int kTileTok = 64;                 // rows per ring stage (4 pages)
+constexpr int kRowsPerWarp = kTileTok / kWarps;
+constexpr float kRescaleThreshold = 16.f;    // log2 units a score may exceed the reference max by
+constexpr long long kWaitCycles = 2000000000ll;
+
+constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
+
+struct TileDesc {
+    int32_t flags;
+    int32_t rows;         // valid rows in this tile
+    int32_t out_row;      // global token row of the item
+    int32_t kv_head;
+    int32_t partial_row;  // -1: final output
+    int32_t pad[3];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag) if the phase did not complete in time
+// or if another thread already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status, int code) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
+
+// Transposing reduction over the LPR lanes that share a row: starts with N values per lane that
+// must each be summed over the lanes; every stage halves the number of values a lane keeps (while
+// more than one is left) and adds the partner's copy.  Afterwards lane `sub` holds the complete
+// sums of values [sub*N/LPR, (sub+1)*N/LPR) (or value sub >> log2(LPR/N) when N < LPR).
+template <int N, int OFF, int NMAX>
+__device__ __forceinline__ void transpose_reduce(float (&v)[NMAX], int lane) {
+    if constexpr (OFF >= 1) {
+        if constexpr (N > 1) {
+            const bool upper = (lane & OFF) != 0;
+#pragma unroll
+            for (int j = 0; j < N / 2; ++j) {
+                const float send = upper ? v[j] : v[j + N / 2];
+                const float keep = upper ? v[j + N / 2] : v[j];
+                v[j] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);
+            }
+            transpose_reduce<N / 2, OFF / 2, NMAX>(v, lane);
+        } else {
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], OFF);
+            transpose_reduce<1, OFF / 2, NMAX>(v, lane);
+        }
+    }
+}
+
+constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
+
+template <int D, int G>
+struct Geometry {
+    static constexpr int LPR = D / 8;                 // lanes per row (16 bytes each)
+    static constexpr int TPW = 32 / LPR;              // rows per warp-wide shared-memory load
+    static constexpr int NR = kRowsPerWarp / TPW;     // rows per lane
+    static constexpr int NV = NR * G;                 // partial dot products per lane
+    static constexpr int NF = NV >= LPR ? NV / LPR : 1;              // finished scores per lane
+    static constexpr int DUP_SHIFT = NV >= LPR ? 0 : ilog2(LPR / NV); // lanes holding duplicates
+    static constexpr int PAGE_BYTES = kPage * D * 2;
+    static constexpr int TILE_BYTES = (kTileTok / kPage) * PAGE_BYTES;   // K (or V) part of a stage
+    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    static constexpr int Q_BYTES = G * D * 2;
+    static constexpr int MERGE_FLOATS = kWarps * G * (D + 2);            // one merge buffer
+    // lane (within a row group) and slot that hold the score of (row i of the lane, head g)
+    __host__ __device__ static constexpr int src_sub(int i, int g) {
+        return NV >= LPR ? (i * G + g) / NF : (i * G + g) << DUP_SHIFT;
+    }
+    __host__ __device__ static constexpr int src_slot(int i, int g) { return NV >= LPR ? (i * G + g) % NF : 0; }
+};
+
+template <int D, int G>
+size_t smem_bytes(int stages) {
+    using Geo = Geometry<D, G>;
+    return (size_t)stages * (Geo::STAGE_BYTES + Geo::Q_BYTES + sizeof(TileDesc) + 16) +
+           2 * Geo::MERGE_FLOATS * sizeof(float) + 3 * 8 + 16 + 1024;
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
+                   const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out,
+                   float* __restrict__ lse, int S) {
+    using Geo = Geometry<D, G>;
+    constexpr int LPR = Geo::LPR, TPW = Geo::TPW, NR = Geo::NR, NV = Geo::NV, NF = Geo::NF;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* stage_base = smem;
+    uint8_t* q_base = stage_base + (size_t)S * Geo::STAGE_BYTES;
+    float* merge_base = (float*)(q_base + (size_t)S * Geo::Q_BYTES);
+    TileDesc* desc = (TileDesc*)(merge_base + 2 * Geo::MERGE_FLOATS);
+    uint64_t* bars = (uint64_t*)(desc + S);      // full[S], empty[S], merge[2]
+    volatile int* abort_flag = (volatile int*)(bars + 2 * S + 2);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), mbar0 = smem_u32(bars + 2 * S);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, kWarps);
+        }
+        mbar_init(mbar0, kWarps);
+        mbar_init(mbar0 + 8, kWarps);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+
+    if (warp == kWarps) {
+        // ------------------------------------------------------------------ producer warp
+        int n = 0;
+        const int i0 = p.cta_indptr_cuda[blockIdx.x], i1 = p.cta_indptr_cuda[blockIdx.x + 1];
+        bool ok = true;
+        for (int ii = i0; ii < i1 && ok; ++ii) {
+            const Item it = p.items[ii];
+            const Unit u = p.units[it.unit];
+            const int kv_end = min(it.kv1, u.kv_limit0);
+            const int partial_row = u.partial_base < 0 ? -1 : u.partial_base + it.chunk;
+            for (int base = it.kv0; base < kv_end; base += kTileTok, ++n) {
+                const int s = n % S;
+                const uint32_t ph = (uint32_t)(n / S) & 1u;
+                ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1);
+                if (!ok) break;
+                const int rows = min(kTileTok, kv_end - base);
+                const int npages = (rows + kPage - 1) / kPage;
+                const bool first = base == it.kv0;
+                if (lane == 0) {
+                    TileDesc d;
+                    d.flags = (first ? kFlagFirst : 0) | (base + kTileTok >= kv_end ? kFlagLast : 0);
+                    d.rows = rows;
+                    d.out_row = u.q_row0;
+                    d.kv_head = u.kv_head;
+                    d.partial_row = partial_row;
+                    desc[s] = d;
+                    mbar_arrive_expect_tx(full0 + 8 * s,
+                                          (uint32_t)(npages * 2 * Geo::PAGE_BYTES + (first ? Geo::Q_BYTES : 0)));
+                }
+                __syncwarp();
+                if (lane < npages) {
+                    const int64_t page = __ldg(p.page_indices + u.page_base + base / kPage + lane);
+                    const __nv_bfloat16* src = pool + pool_row_offset(page, 0, u.kv_head, 0, Hkv, D);
+                    const uint32_t dst = smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * Geo::PAGE_BYTES);
+                    bulk_g2s(dst, src, Geo::PAGE_BYTES, full0 + 8 * s);
+                    bulk_g2s(dst + Geo::TILE_BYTES, src + (size_t)Hkv * kPage * D, Geo::PAGE_BYTES, full0 + 8 * s);
+                }
+                if (first && lane == 31) {
+                    const __nv_bfloat16* src = q + ((size_t)u.q_row0 * Hq + (size_t)u.kv_head * G) * D;
+                    bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
+                }
+            }
+        }
+        if (ok) {
+            const int s = n % S;
+            const uint32_t ph = (uint32_t)(n / S) & 1u;
+            if (mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1)) {
+                if (lane == 0) {
+                    desc[s].flags = kFlagEnd;
+                    mbar_arrive(full0 + 8 * s);
+                }
+            }
+        } else {
+            // aborted: let the copies already issued land before the CTA's shared memory goes away
+            const long long t0 = clock64();
+            for (int k = max(0, n - S); k < n; ++k)
+                while (!mbar_try_wait(full0 + 8 * (k % S), (uint32_t)(k / S) & 1u) &&
+                       clock64() - t0 < kWaitCycles) {}
+        }
+        return;
+    }
+
+    // ---------------------------------------------------------------------- consumer warps
+    const int sub = lane % LPR;
+    const int grp = lane / LPR;
+    const int my_row = (sub >> 2) * TPW + grp;   // row (within the warp's 8) of this lane's scores
+    const float qscale = p.sm_scale * kLog2e;
+
+    float2 q2[G][4];
+    float2 o2[G][4];
+    float m_ref[G];
+    float m_own[NF], l_own[NF];
+    int item_count = 0;
+    int32_t cur_out_row = 0, cur_kv_head = 0, cur_partial = -1;
+
+    for (int n = 0;; ++n) {
+        const int s = n % S;
+        const uint32_t ph = (uint32_t)(n / S) & 1u;
+        if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status, 2)) break;
+        const TileDesc d = desc[s];
+        if (d.flags & kFlagEnd) break;
+        if (d.flags & kFlagFirst) {
+            const uint8_t* qs = q_base + (size_t)s * Geo::Q_BYTES;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const uint4 w = *reinterpret_cast<const uint4*>(qs + ((size_t)g * D + sub * 8) * 2);
+                q2[g][0] = unpack2(w.x); q2[g][1] = unpack2(w.y);
+                q2[g][2] = unpack2(w.z); q2[g][3] = unpack2(w.w);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    q2[g][j].x *= qscale; q2[g][j].y *= qscale;
+                    o2[g][j] = make_float2(0.f, 0.f);
+                }
+                m_ref[g] = -INFINITY;
+            }
+#pragma unroll
+            for (int f = 0; f < NF; ++f) { m_own[f] = -INFINITY; l_own[f] = 0.f; }
+            cur_out_row = d.out_row; cur_kv_head = d.kv_head; cur_partial = d.partial_row;
+        }
+        const int rows = d.rows;
+        const bool active = warp * kRowsPerWarp < rows;
+        uint4 kw[NR], vw[NR];
+        if (active) {
+            const uint8_t* ks = stage_base + (size_t)s * Geo::STAGE_BYTES +
+                                (size_t)(warp * kRowsPerWarp) * (D * 2) + lane * 16;
+#pragma unroll
+            for (int i = 0; i < NR; ++i) {
+                kw[i] = *reinterpret_cast<const uint4*>(ks + (size_t)i * TPW * D * 2);
+                vw[i] = *reinterpret_cast<const uint4*>(ks + Geo::TILE_BYTES + (size_t)i * TPW * D * 2);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty0 + 8 * s);
+
+        if (active) {
+            const bool tail = rows < (warp + 1) * kRowsPerWarp;
+            if (tail) {
+#pragma unroll
+                for (int i = 0; i < NR; ++i)
+                    if (warp * kRowsPerWarp + i * TPW + grp >= rows) {
+                        kw[i] = make_uint4(0, 0, 0, 0);
+                        vw[i] = make_uint4(0, 0, 0, 0);
+                    }
+            }
+            // scores: partial dot products over this lane's 8 elements, then reduce over the row's lanes
+            float v[NV];
+#pragma unroll
+            for (int i = 0; i < NR; ++i) {
+                const float2 k0 = unpack2(kw[i].x), k1 = unpack2(kw[i].y), k2 = unpack2(kw[i].z), k3 = unpack2(kw[i].w);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float2 a = __fmul2_rn(q2[g][0], k0);
+                    a = __ffma2_rn(q2[g][1], k1, a);
+                    a = __ffma2_rn(q2[g][2], k2, a);
+                    a = __ffma2_rn(q2[g][3], k3, a);
+                    v[i * G + g] = a.x + a.y;
+                }
+            }
+            transpose_reduce<NV, LPR / 2, NV>(v, lane);
+            float sc[NF];
+#pragma unroll
+            for (int f = 0; f < NF; ++f) sc[f] = v[f];
+            if (tail && warp * kRowsPerWarp + my_row >= rows) {
+#pragma unroll
+                for (int f = 0; f < NF; ++f) sc[f] = -INFINITY;
+            }
+            bool need = false;
+#pragma unroll
+            for (int f = 0; f < NF; ++f) need |= sc[f] > m_own[f] + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {
+                // move the reference maximum: per head, over this warp's rows of the tile
+                float mn[NF];
+#pragma unroll
+                for (int f = 0; f < NF; ++f) {
+                    float t = sc[f];
+                    t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 4));
+                    t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 8));
+                    t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 16));
+                    mn[f] = fmaxf(m_own[f], t);
+                }
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const float mg = __shfl_sync(0xffffffffu, mn[Geo::src_slot(0, g)], Geo::src_sub(0, g));
+                    const float scale = fast_exp2(m_ref[g] - mg);
+                    m_ref[g] = mg;
+                    const float2 s2 = make_float2(scale, scale);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) o2[g][j] = __fmul2_rn(o2[g][j], s2);
+                }
+#pragma unroll
+                for (int f = 0; f < NF; ++f) {
+                    l_own[f] *= fast_exp2(m_own[f] - mn[f]);
+                    m_own[f] = mn[f];
+                }
+            }
+            float pr[NF];
+#pragma unroll
+            for (int f = 0; f < NF; ++f) {
+                pr[f] = fast_exp2(sc[f] - m_own[f]);
+                l_own[f] += pr[f];
+            }
+#pragma unroll
+            for (int i = 0; i < NR; ++i) {
+                const float2 v0 = unpack2(vw[i].x), v1 = unpack2(vw[i].y), v2 = unpack2(vw[i].z), v3 = unpack2(vw[i].w);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const float pg = __shfl_sync(0xffffffffu, pr[Geo::src_slot(i, g)],
+                                                 grp * LPR + Geo::src_sub(i, g));
+                    const float2 pp = make_float2(pg, pg);
+                    o2[g][0] = __ffma2_rn(pp, v0, o2[g][0]);
+                    o2[g][1] = __ffma2_rn(pp, v1, o2[g][1]);
+                    o2[g][2] = __ffma2_rn(pp, v2, o2[g][2]);
+                    o2[g][3] = __ffma2_rn(pp, v3, o2[g][3]);
+                }
+            }
+        }
+
+        if (d.flags & kFlagLast) {
+            // ---- end of item: merge the warps' states and write the result
+            float* mm = merge_base + (size_t)(item_count & 1) * Geo::MERGE_FLOATS;   // [warp][G] max
+            float* ml = mm + kWarps * G;                                          // [warp][G] sum
+            float* mo = ml + kWarps * G;                                          // [warp][G][D]
+#pragma unroll
+            for (int f = 0; f < NF; ++f) {
+                l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 4);
+                l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 8);
+                l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 16);
+            }
+#pragma unroll
+            for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        o2[g][j].x += __shfl_xor_sync(0xffffffffu, o2[g][j].x, off);
+                        o2[g][j].y += __shfl_xor_sync(0xffffffffu, o2[g][j].y, off);
+                    }
+            if (grp == 0) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float4* dst = reinterpret_cast<float4*>(mo + ((size_t)warp * G + g) * D + sub * 8);
+                    dst[0] = make_float4(o2[g][0].x, o2[g][0].y, o2[g][1].x, o2[g][1].y);
+                    dst[1] = make_float4(o2[g][2].x, o2[g][2].y, o2[g][3].x, o2[g][3].y);
+                }
+                if ((sub >> 2) == 0) {
+#pragma unroll
+                    for (int f = 0; f < NF; ++f) {
+                        const int k = NV >= LPR ? sub * NF + f : sub >> Geo::DUP_SHIFT;
+                        const int g = k % G;
+                        mm[warp * G + g] = m_own[f];
+                        ml[warp * G + g] = l_own[f];
+                    }
+                }
+            }
+            __syncwarp();
+            const int buf = item_count & 1;
+            const uint32_t mb = mbar0 + 8 * buf;
+            if (lane == 0) mbar_arrive(mb);
+            // barrier `buf` serves every second item; its phase flips once per use
+            if (!mbar_wait(mb, (uint32_t)(item_count >> 1) & 1u, abort_flag, p.status, 3)) break;
+            ++item_count;
+            const int tid = threadIdx.x;
+            for (int e = 2 * tid; e < G * D; e += 2 * kWarps * 32) {
+                const int g = e / D, dd = e % D;
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mm[w * G + g]);
+                float L = 0.f, a0 = 0.f, a1 = 0.f;
+#pragma unroll
+                for (int w = 0; w < kWarps; ++w) {
+                    const float wgt = fast_exp2(mm[w * G + g] - M);
+                    L = fmaf(ml[w * G + g], wgt, L);
+                    const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * G + g) * D + dd);
+                    a0 = fmaf(ov.x, wgt, a0);
+                    a1 = fmaf(ov.y, wgt, a1);
+                }
+                const float inv = 1.f / L;
+                const size_t hq = (size_t)cur_kv_head * G + g;
+                if (cur_partial < 0) {
+                    *reinterpret_cast<uint32_t*>(out + ((size_t)cur_out_row * Hq + hq) * D + dd) =
+                        pack_bf16x2(a0 * inv, a1 * inv);
+                    if (lse != nullptr && dd == 0)
+                        lse[(size_t)cur_out_row * Hq + hq] = (M + log2f(L)) * kLn2;
+                } else {
+                    *reinterpret_cast<float2*>(p.partial_o + ((size_t)cur_partial * G + g) * D + dd) =
+                        make_float2(a0 * inv, a1 * inv);
+                    if (dd == 0) p.partial_lse[(size_t)cur_partial * G + g] = M + log2f(L);
+                }
+            }
+        }
+    }
+}
+
+template <int D, int G>
+static cudaError_t launch_dg(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
+                             cudaStream_t stream) {
+    int S = 8;
+    while (S > 2 && smem_bytes<D, G>(S) > 232448) --S;
+    const size_t smem = smem_bytes<D, G>(S);
+    cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attn_decode_kernel<D, G><<<p.num_ctas_cuda, kThreads, smem, stream>>>(
+        p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t launch_d(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
+                            cudaStream_t stream) {
+    switch (p.group) {
+        case 1: return launch_dg<D, 1>(p, q, pool, out, lse, stream);
+        case 2: return launch_dg<D, 2>(p, q, pool, out, lse, stream);
+        case 4: return launch_dg<D, 4>(p, q, pool, out, lse, stream);
+        case 8: return launch_dg<D, 8>(p, q, pool, out, lse, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace dec
+
+cudaError_t launch_attn_decode(const DevPlan& p, const void* q, const void* kv_pool, void* out,
+                               float* lse, cudaStream_t stream) {
+    if (p.num_items_cuda == 0) return cudaSuccess;
+    if (p.head_dim == 128) return dec::launch_d<128>(p, q, kv_pool, out, lse, stream);
+    if (p.head_dim == 64) return dec::launch_d<64>(p, q, kv_pool, out, lse, stream);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace asynclm

@@ -9,8 +9,8 @@ namespace asynclm {
 cudaError_t launch_kv_append(const DevPlan& p, const void* k_new, const void* v_new, void* kv_pool,
                              cudaStream_t stream);
 
-cudaError_t launch_attn_cuda_core(const DevPlan& p, const void* q, const void* kv_pool, void* out,
-                                  float* lse, cudaStream_t stream);
+cudaError_t launch_attn_decode(const DevPlan& p, const void* q, const void* kv_pool, void* out,
+                               float* lse, cudaStream_t stream);
 
 cudaError_t launch_lse_merge(const DevPlan& p, void* out, float* lse, cudaStream_t stream);
 

@@ -9,8 +9,8 @@ namespace asynclm {
 
 constexpr uint64_t kPlanMagic = 0x4153594e434c4d31ull;   // "ASYNCLM1"
 
-// Persistent warp slots per SM of the CUDA-core attention kernel.
-constexpr int kCudaSlotsPerSm = 16;
+// Persistent CTAs per SM of the CUDA-core attention kernel.
+constexpr int kCudaSlotsPerSm = 1;
 // Fixed cost of starting an item, in units of one 128-token KV tile, used when balancing CTAs.
 constexpr int kCudaItemOverheadTiles = 1;
 constexpr int kTensorItemOverheadTiles = 1;
