@@ -50,7 +50,9 @@ typedef enum asynclm_status {
     ASYNCLM_ERR_WORKSPACE_TOO_SMALL = -4,
     ASYNCLM_ERR_CUDA = -5,                /* a CUDA runtime call or a launch failed            */
     ASYNCLM_ERR_ARCH = -6,                /* current device is not compute capability 10.x     */
-    ASYNCLM_ERR_DEVICE_STATUS = -7        /* a kernel reported a bounded wait that ran out     */
+    ASYNCLM_ERR_DEVICE_STATUS = -7,       /* a kernel reported a bounded wait that ran out     */
+    ASYNCLM_ERR_STATIC_SCRATCH_TOO_SMALL = -8  /* asynclm_attn_mixed_static: the plan's partial
+                                             results exceed ASYNCLM_STATIC_SCRATCH_BYTES         */
 } asynclm_status;
 
 /* Supported: head_dim in {64, 128}; page_size = 16; num_q_heads / num_kv_heads in {1, 2, 4, 8}. */
@@ -207,6 +209,43 @@ int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv
  * ASYNCLM_OK or ASYNCLM_ERR_DEVICE_STATUS / ASYNCLM_ERR_CUDA.
  */
 int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out);
+
+/*
+ * asynclm_attn_mixed with no caller-provided scratch (the paper has no counterpart to this call; it
+ * exists for deployment reasons only).
+ *
+ * Some callers cannot allocate device memory for the library: a server that gave all of HBM to
+ * its KV pool and weights at start-up, a plug-in that may not touch its host's memory pool, a
+ * latency-critical loop in which cudaMalloc is banned because it can stall the device.  For them
+ * the fp32 partial results of split contexts (the only scratch the attention kernels use) are kept
+ * in a fixed array of ASYNCLM_STATIC_SCRATCH_BYTES that is compiled into the library; every GPU
+ * that uses the library holds that array until the process exits.  The call itself performs no
+ * allocation and no free, on the device or through any library.
+ *
+ * Arguments, results and numerics are exactly those of asynclm_attn_mixed, computed by the same
+ * kernels.  The plan's device workspace is still the caller's (it holds the uploaded plan), but
+ * the part of it reserved for partial results is left unused.
+ *
+ *   - A plan whose partial results need more than ASYNCLM_STATIC_SCRATCH_BYTES
+ *     (align256(partial_rows * G * head_dim * 4) + align256(partial_rows * G * 4), with
+ *     partial_rows from asynclm_plan_get_info) is refused with
+ *     ASYNCLM_ERR_STATIC_SCRATCH_TOO_SMALL before anything is launched; plan with a longer
+ *     kv_chunk_tokens, or use asynclm_attn_mixed.
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress with that device current).  Make that first call before starting any
+ *     stream capture on that device.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left in
+ *     it.  Nothing in it has to start at zero: each call writes every partial row before reading
+ *     it.  Two calls whose kernels may overlap on the GPU (different streams, or different threads
+ *     or processes' streams of one process image) race on the array; run them on one stream or
+ *     order them with events.
+ * Errors: INVALID_ARG, STATIC_SCRATCH_TOO_SMALL, CUDA.
+ */
+#define ASYNCLM_STATIC_SCRATCH_BYTES (16u << 20)
+int asynclm_attn_mixed_static(const asynclm_plan_t* plan, const void* q, const void* kv_pool,
+                              void* out, float* lse, void* stream);
+/* The compiled-in value of ASYNCLM_STATIC_SCRATCH_BYTES. */
+size_t asynclm_static_scratch_bytes(void);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,8 @@ from . import build as _build
 EXPORTS = [
     "asynclm_version", "asynclm_strerror", "asynclm_plan_workspace_size", "asynclm_plan",
     "asynclm_plan_get_info", "asynclm_plan_get_items", "asynclm_kv_append", "asynclm_attn_mixed",
-    "asynclm_last_device_status", "asynclm_last_cuda_error",
+    "asynclm_last_device_status", "asynclm_last_cuda_error", "asynclm_attn_mixed_static",
+    "asynclm_static_scratch_bytes",
 ]
 
 PLAN_REJECT_ALIASED_WRITES = 1
@@ -96,10 +97,13 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_plan_get_items.argtypes = [vp, vp, i32]
     lib.asynclm_kv_append.argtypes = [vp, vp, vp, vp, vp]
     lib.asynclm_attn_mixed.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.asynclm_attn_mixed_static.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.asynclm_static_scratch_bytes.argtypes = []
     lib.asynclm_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     for name in EXPORTS:
-        if name not in ("asynclm_strerror", "asynclm_last_cuda_error"):
+        if name not in ("asynclm_strerror", "asynclm_last_cuda_error", "asynclm_static_scratch_bytes"):
             getattr(lib, name).restype = ctypes.c_int
+    lib.asynclm_static_scratch_bytes.restype = ctypes.c_size_t
     _lib = lib
     return lib
 
@@ -234,6 +238,18 @@ def asynclm_attn_mixed(plan: Plan, q, kv_pool, out, lse=None, stream=None) -> No
     _check(load().asynclm_attn_mixed(plan.handle, q.data_ptr(), kv_pool.data_ptr(), out.data_ptr(),
                                      None if lse is None else lse.data_ptr(), _stream_ptr(stream)),
            "asynclm_attn_mixed")
+
+
+def asynclm_attn_mixed_static(plan: Plan, q, kv_pool, out, lse=None, stream=None) -> None:
+    """asynclm_attn_mixed for callers that cannot hand the library scratch memory: split-KV
+    partial results go to the fixed array inside the library (see include/asynclm.h)."""
+    _check(load().asynclm_attn_mixed_static(plan.handle, q.data_ptr(), kv_pool.data_ptr(),
+                                            out.data_ptr(), None if lse is None else lse.data_ptr(),
+                                            _stream_ptr(stream)), "asynclm_attn_mixed_static")
+
+
+def static_scratch_bytes() -> int:
+    return int(load().asynclm_static_scratch_bytes())
 
 
 def last_device_status(plan: Plan, stream=None) -> int:

@@ -34,6 +34,8 @@ extern "C" const char* asynclm_strerror(int status) {
         case ASYNCLM_ERR_CUDA: return "CUDA runtime error";
         case ASYNCLM_ERR_ARCH: return "device is not compute capability 10.x";
         case ASYNCLM_ERR_DEVICE_STATUS: return "a kernel reported a bounded wait that ran out";
+        case ASYNCLM_ERR_STATIC_SCRATCH_TOO_SMALL:
+            return "the plan's split-KV partial results do not fit the library's fixed scratch array";
         default: return "unknown status";
     }
 }
