@@ -86,25 +86,25 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 
 __device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
 
-// Transposing reduction over the LPR lanes that share a row: starts with N values per lane that
-// must each be summed over the lanes; every stage halves the number of values a lane keeps (while
-// more than one is left) and adds the partner's copy.  Afterwards lane `sub` holds the complete
-// sums of values [sub*N/LPR, (sub+1)*N/LPR) (or value sub >> log2(LPR/N) when N < LPR).
+// Transposing reduction over the LPR lanes that share a row.  Every lane starts with N values that
+// must each be summed over the LPR lanes; each stage halves the number of values a lane keeps
+// (while more than one is left) and adds the partner's copy of the kept half.  No selects are
+// needed because a lane fills its slots in a lane-dependent order: slot k of lane `sub` holds the
+// value with true index k ^ mask(sub), mask(sub) = sub * N / LPR (or sub >> log2(LPR / N) when
+// N < LPR), so at every stage all lanes keep the lower half of their slots and send the upper
+// half.  Afterwards slot f of lane `sub` holds the complete sum of true index
+// sub * (N / LPR) + f (or sub >> log2(LPR / N) when N < LPR, duplicated over neighbouring lanes).
 template <int N, int OFF, int NMAX>
-__device__ __forceinline__ void transpose_reduce(float (&v)[NMAX], int lane) {
+__device__ __forceinline__ void transpose_reduce(float (&v)[NMAX]) {
     if constexpr (OFF >= 1) {
         if constexpr (N > 1) {
-            const bool upper = (lane & OFF) != 0;
 #pragma unroll
-            for (int j = 0; j < N / 2; ++j) {
-                const float send = upper ? v[j] : v[j + N / 2];
-                const float keep = upper ? v[j + N / 2] : v[j];
-                v[j] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);
-            }
-            transpose_reduce<N / 2, OFF / 2, NMAX>(v, lane);
+            for (int j = 0; j < N / 2; ++j)
+                v[j] += __shfl_xor_sync(0xffffffffu, v[j + N / 2], OFF);
+            transpose_reduce<N / 2, OFF / 2, NMAX>(v);
         } else {
             v[0] += __shfl_xor_sync(0xffffffffu, v[0], OFF);
-            transpose_reduce<1, OFF / 2, NMAX>(v, lane);
+            transpose_reduce<1, OFF / 2, NMAX>(v);
         }
     }
 }
@@ -124,11 +124,14 @@ struct Geometry {
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
     static constexpr int Q_BYTES = G * D * 2;
     static constexpr int MERGE_FLOATS = kWarps * G * (D + 2);            // one merge buffer
-    // lane (within a row group) and slot that hold the score of (row i of the lane, head g)
-    __host__ __device__ static constexpr int src_sub(int i, int g) {
+    // A lane's slot (i, g) holds the partial score of true row i ^ xi and true head g ^ xg, with
+    // (xi, xg) = (mask / G, mask % G) and mask as in transpose_reduce.  The finished score of a
+    // lane's slot (i, g) sits in slot score_slot(i, g) of the lane whose index differs from its own
+    // by score_xor(i, g).
+    __host__ __device__ static constexpr int score_xor(int i, int g) {
         return NV >= LPR ? (i * G + g) / NF : (i * G + g) << DUP_SHIFT;
     }
-    __host__ __device__ static constexpr int src_slot(int i, int g) { return NV >= LPR ? (i * G + g) % NF : 0; }
+    __host__ __device__ static constexpr int score_slot(int i, int g) { return NV >= LPR ? (i * G + g) % NF : 0; }
 };
 
 template <int D, int G>
@@ -175,46 +178,81 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
 
     if (warp == kWarps) {
         // ------------------------------------------------------------------ producer warp
+        // The page ids of the next 32 pages (8 tiles) and the descriptors of the next two items are
+        // fetched ahead of use, so that no global-load latency sits between two tiles.
+        struct PItem { int kv0, kv_end, q_row0, kv_head, partial_row, page0; };
         int n = 0;
         const int i0 = p.cta_indptr_cuda[blockIdx.x], i1 = p.cta_indptr_cuda[blockIdx.x + 1];
-        bool ok = true;
-        for (int ii = i0; ii < i1 && ok; ++ii) {
-            const Item it = p.items[ii];
-            const Unit u = p.units[it.unit];
-            const int kv_end = min(it.kv1, u.kv_limit0);
-            const int partial_row = u.partial_base < 0 ? -1 : u.partial_base + it.chunk;
-            for (int base = it.kv0; base < kv_end; base += kTileTok, ++n) {
-                const int s = n % S;
-                const uint32_t ph = (uint32_t)(n / S) & 1u;
-                ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1);
-                if (!ok) break;
-                const int rows = min(kTileTok, kv_end - base);
-                const int npages = (rows + kPage - 1) / kPage;
-                const bool first = base == it.kv0;
-                if (lane == 0) {
-                    TileDesc d;
-                    d.flags = (first ? kFlagFirst : 0) | (base + kTileTok >= kv_end ? kFlagLast : 0);
-                    d.rows = rows;
-                    d.out_row = u.q_row0;
-                    d.kv_head = u.kv_head;
-                    d.partial_row = partial_row;
-                    desc[s] = d;
-                    mbar_arrive_expect_tx(full0 + 8 * s,
-                                          (uint32_t)(npages * 2 * Geo::PAGE_BYTES + (first ? Geo::Q_BYTES : 0)));
-                }
-                __syncwarp();
-                if (lane < npages) {
-                    const int64_t page = __ldg(p.page_indices + u.page_base + base / kPage + lane);
-                    const __nv_bfloat16* src = pool + pool_row_offset(page, 0, u.kv_head, 0, Hkv, D);
-                    const uint32_t dst = smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * Geo::PAGE_BYTES);
-                    bulk_g2s(dst, src, Geo::PAGE_BYTES, full0 + 8 * s);
-                    bulk_g2s(dst + Geo::TILE_BYTES, src + (size_t)Hkv * kPage * D, Geo::PAGE_BYTES, full0 + 8 * s);
-                }
-                if (first && lane == 31) {
-                    const __nv_bfloat16* src = q + ((size_t)u.q_row0 * Hq + (size_t)u.kv_head * G) * D;
-                    bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
-                }
+        auto load_item = [&](int ii) {
+            PItem r{0, 0, 0, 0, -1, 0};
+            if (ii < i1) {
+                const Item it = p.items[ii];
+                const Unit u = p.units[it.unit];
+                r.kv0 = it.kv0;
+                r.kv_end = min(it.kv1, u.kv_limit0);
+                r.q_row0 = u.q_row0;
+                r.kv_head = u.kv_head;
+                r.partial_row = u.partial_base < 0 ? -1 : u.partial_base + it.chunk;
+                r.page0 = u.page_base + it.kv0 / kPage;
             }
+            return r;
+        };
+        auto load_pages = [&](const PItem& it, int first_page) {
+            const int npg = (it.kv_end - it.kv0 + kPage - 1) / kPage;
+            const int idx = first_page + lane;
+            return idx < npg ? __ldg(p.page_indices + it.page0 + idx) : 0;
+        };
+        constexpr int kPagesPerTile = kTileTok / kPage;
+        constexpr int kGroupTiles = 32 / kPagesPerTile;
+        bool ok = true;
+        PItem cur = load_item(i0), nxt = load_item(i0 + 1);
+        int pages_cur = cur.kv_end > 0 ? load_pages(cur, 0) : 0;
+        for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
+            const PItem after = load_item(ii + 2);
+            const int ntiles = (cur.kv_end - cur.kv0 + kTileTok - 1) / kTileTok;
+            for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
+                int pages_nxt = 0;
+                if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
+                else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
+                const int t1 = min(t0 + kGroupTiles, ntiles);
+                for (int t = t0; t < t1; ++t, ++n) {
+                    const int s = n % S;
+                    const uint32_t ph = (uint32_t)(n / S) & 1u;
+                    ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, p.status, 1);
+                    if (!ok) break;
+                    const int base = cur.kv0 + t * kTileTok;
+                    const int rows = min(kTileTok, cur.kv_end - base);
+                    const int npages = (rows + kPage - 1) / kPage;
+                    const bool first = t == 0;
+                    if (lane == 0) {
+                        TileDesc d;
+                        d.flags = (first ? kFlagFirst : 0) | (t == ntiles - 1 ? kFlagLast : 0);
+                        d.rows = rows;
+                        d.out_row = cur.q_row0;
+                        d.kv_head = cur.kv_head;
+                        d.partial_row = cur.partial_row;
+                        desc[s] = d;
+                        mbar_arrive_expect_tx(full0 + 8 * s,
+                                              (uint32_t)(npages * 2 * Geo::PAGE_BYTES + (first ? Geo::Q_BYTES : 0)));
+                    }
+                    __syncwarp();
+                    const int64_t page = __shfl_sync(0xffffffffu, pages_cur,
+                                                     (t - t0) * kPagesPerTile + (lane & (kPagesPerTile - 1)));
+                    if (lane < npages) {
+                        const __nv_bfloat16* src = pool + pool_row_offset(page, 0, cur.kv_head, 0, Hkv, D);
+                        const uint32_t dst = smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * Geo::PAGE_BYTES);
+                        bulk_g2s(dst, src, Geo::PAGE_BYTES, full0 + 8 * s);
+                        bulk_g2s(dst + Geo::TILE_BYTES, src + (size_t)Hkv * kPage * D, Geo::PAGE_BYTES, full0 + 8 * s);
+                    }
+                    if (first && lane == 31) {
+                        const __nv_bfloat16* src = q + ((size_t)cur.q_row0 * Hq + (size_t)cur.kv_head * G) * D;
+                        bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
+                    }
+                }
+                pages_cur = pages_nxt;
+            }
+            cur = nxt;
+            nxt = after;
         }
         if (ok) {
             const int s = n % S;
@@ -239,6 +277,9 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     const int sub = lane % LPR;
     const int grp = lane / LPR;
     const int my_row = (sub >> 2) * TPW + grp;   // row (within the warp's 8) of this lane's scores
+    const int mask = NV >= LPR ? sub * NF : sub >> Geo::DUP_SHIFT;
+    const int xi = mask / G;                     // this lane's slot i holds true row i ^ xi
+    const int xg = mask % G;                     // and its slot g holds true head g ^ xg
     const float qscale = p.sm_scale * kLog2e;
 
     float2 q2[G][4];
@@ -258,7 +299,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             const uint8_t* qs = q_base + (size_t)s * Geo::Q_BYTES;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const uint4 w = *reinterpret_cast<const uint4*>(qs + ((size_t)g * D + sub * 8) * 2);
+                const uint4 w = *reinterpret_cast<const uint4*>(qs + ((size_t)(g ^ xg) * D + sub * 8) * 2);
                 q2[g][0] = unpack2(w.x); q2[g][1] = unpack2(w.y);
                 q2[g][2] = unpack2(w.z); q2[g][3] = unpack2(w.w);
 #pragma unroll
@@ -280,8 +321,8 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
                                 (size_t)(warp * kRowsPerWarp) * (D * 2) + lane * 16;
 #pragma unroll
             for (int i = 0; i < NR; ++i) {
-                kw[i] = *reinterpret_cast<const uint4*>(ks + (size_t)i * TPW * D * 2);
-                vw[i] = *reinterpret_cast<const uint4*>(ks + Geo::TILE_BYTES + (size_t)i * TPW * D * 2);
+                kw[i] = *reinterpret_cast<const uint4*>(ks + (size_t)(i ^ xi) * TPW * D * 2);
+                vw[i] = *reinterpret_cast<const uint4*>(ks + Geo::TILE_BYTES + (size_t)(i ^ xi) * TPW * D * 2);
             }
         }
         __syncwarp();
@@ -292,7 +333,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             if (tail) {
 #pragma unroll
                 for (int i = 0; i < NR; ++i)
-                    if (warp * kRowsPerWarp + i * TPW + grp >= rows) {
+                    if (warp * kRowsPerWarp + (i ^ xi) * TPW + grp >= rows) {
                         kw[i] = make_uint4(0, 0, 0, 0);
                         vw[i] = make_uint4(0, 0, 0, 0);
                     }
@@ -311,7 +352,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
                     v[i * G + g] = a.x + a.y;
                 }
             }
-            transpose_reduce<NV, LPR / 2, NV>(v, lane);
+            transpose_reduce<NV, LPR / 2, NV>(v);
             float sc[NF];
 #pragma unroll
             for (int f = 0; f < NF; ++f) sc[f] = v[f];
@@ -335,7 +376,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
                 }
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    const float mg = __shfl_sync(0xffffffffu, mn[Geo::src_slot(0, g)], Geo::src_sub(0, g));
+                    const float mg = __shfl_xor_sync(0xffffffffu, mn[Geo::score_slot(0, g)], Geo::score_xor(0, g));
                     const float scale = fast_exp2(m_ref[g] - mg);
                     m_ref[g] = mg;
                     const float2 s2 = make_float2(scale, scale);
@@ -359,8 +400,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
                 const float2 v0 = unpack2(vw[i].x), v1 = unpack2(vw[i].y), v2 = unpack2(vw[i].z), v3 = unpack2(vw[i].w);
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    const float pg = __shfl_sync(0xffffffffu, pr[Geo::src_slot(i, g)],
-                                                 grp * LPR + Geo::src_sub(i, g));
+                    const float pg = __shfl_xor_sync(0xffffffffu, pr[Geo::score_slot(i, g)], Geo::score_xor(i, g));
                     const float2 pp = make_float2(pg, pg);
                     o2[g][0] = __ffma2_rn(pp, v0, o2[g][0]);
                     o2[g][1] = __ffma2_rn(pp, v1, o2[g][1]);
@@ -393,7 +433,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             if (grp == 0) {
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
-                    float4* dst = reinterpret_cast<float4*>(mo + ((size_t)warp * G + g) * D + sub * 8);
+                    float4* dst = reinterpret_cast<float4*>(mo + ((size_t)warp * G + (g ^ xg)) * D + sub * 8);
                     dst[0] = make_float4(o2[g][0].x, o2[g][0].y, o2[g][1].x, o2[g][1].y);
                     dst[1] = make_float4(o2[g][2].x, o2[g][2].y, o2[g][3].x, o2[g][3].y);
                 }
