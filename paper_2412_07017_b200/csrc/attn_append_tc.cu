@@ -1,0 +1,584 @@
+// Tensor-core attention for interrupt spans (tcgen05 MMA with accumulators in tensor memory).
+//
+// An interrupt span is a block of new tokens appended to one sequence (paper Section 3.2); in the
+// next decoding step (Section 5.3) every token of the span attends to the whole cached context and
+// causally to the span itself.  With G query heads per kv head, a span of q tokens gives G*q query
+// rows against the same K/V, which is a dense contraction: rows are packed 128 to a tile
+// (row m = token m / G, head m % G) and S = Q K^T and O += P V run on the tensor cores.
+//
+// One persistent CTA per SM, six warps:
+//   warps 0-3  one thread per query row: Q staging, softmax on S read from tensor memory, P written
+//              to shared memory as bf16, lazy rescaling of O, epilogue
+//   warp 4     producer: tiled TMA loads of K/V pages (16 tokens x 64 values per box, 128-byte
+//              swizzle) into two-stage rings
+//   warp 5     one thread issues the MMAs; the warp owns the tensor-memory allocation
+// S is double buffered in tensor memory so that Q K^T of the next tile runs under the softmax of the
+// current one.  All hand-offs are mbarriers with bounded waits; a wait that runs out sets the plan's
+// status word and a CTA-wide abort flag, every role falls through to the common exit, and the
+// tensor memory is released there.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace asynclm {
+
+namespace tc {
+
+constexpr int kThreads = 192;
+constexpr int kD = 128;
+constexpr int kTile = 128;                       // keys per KV tile and query rows per tile
+constexpr int kKS = 2, kVS = 2;                  // ring depths
+constexpr uint32_t kHalfBytes = 128 * 128;       // one 64-value half of a 128-row tile
+constexpr uint32_t kTileBytes = 2 * kHalfBytes;  // 32 KiB
+constexpr uint32_t kBoxBytes = 16 * 128;         // one TMA box: 16 tokens x 64 values
+constexpr float kRescaleThreshold = 8.f;
+constexpr long long kWaitCycles = 2000000000ll;
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffP = kOffQ + kTileBytes;
+constexpr uint32_t kOffK = kOffP + kTileBytes;
+constexpr uint32_t kOffV = kOffK + kKS * kTileBytes;
+constexpr uint32_t kOffBar = kOffV + kVS * kTileBytes;
+enum Bar { kQFull = 0, kPFull, kPvDone, kOFree, kSFull0, kSFull1, kKFull0, kKEmpty0 = kKFull0 + kKS,
+           kVFull0 = kKEmpty0 + kKS, kVEmpty0 = kVFull0 + kVS, kMmaDrain = kVEmpty0 + kVS, kNumBars };
+constexpr uint32_t kOffTmemPtr = kOffBar + 8 * kNumBars;
+constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
+constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
+
+// tensor memory columns
+constexpr uint32_t kColS = 0;      // two S buffers of 128 columns
+constexpr uint32_t kColO = 256;    // O accumulator, 128 columns
+constexpr uint32_t kTmemCols = 512;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status, int code) {
+    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+    return true;
+}
+// The same wait with a warp-uniform verdict, for code that goes on to warp-collective instructions.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* status, int code) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, code));
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 2-D tiled TMA load (no multicast): box (64 values, 16 rows) at (x, y) of the pool viewed as
+// [rows][128 values].
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+           ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = n; b_mn = 1 when B is stored with N
+// contiguous (the V tile), 0 when K is contiguous.
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, uint32_t b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+#define TC_R32(r) \
+    "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), \
+    "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), \
+    "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), \
+    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+#define TC_W32(r) \
+    "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), \
+    "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), \
+    "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), \
+    "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+
+// This warp's 32 rows x 32 consecutive fp32 columns of tensor memory -> one row per thread.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : TC_R32(r) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+        ::TC_W32(r), "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+struct TItem {
+    int kv0, kv_end;      // key range of the item after causal clipping (kv_end == 0: no item)
+    int q_row0, ntok, kv_limit0, kv_head, partial_base, chunk, page0;
+};
+
+__device__ __forceinline__ TItem load_titem(const DevPlan& p, int ii, int i1) {
+    TItem r{0, 0, 0, 0, 0, 0, -1, 0, 0};
+    if (ii < i1) {
+        const Item it = p.items[ii];
+        const Unit u = p.units[it.unit];
+        r.kv0 = it.kv0;
+        r.kv_end = min(it.kv1, u.kv_limit0 + u.ntok - 1);
+        r.q_row0 = u.q_row0;
+        r.ntok = u.ntok;
+        r.kv_limit0 = u.kv_limit0;
+        r.kv_head = u.kv_head;
+        r.partial_base = u.partial_base;
+        r.chunk = it.chunk;
+        r.page0 = u.page_base + it.kv0 / kPage;
+    }
+    return r;
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
+                      const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
+                      float* __restrict__ lse) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + kOffBar;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    volatile uint32_t* tmem_ptr = (volatile uint32_t*)(smem + kOffTmemPtr);
+    volatile int* abort_flag = (volatile int*)(smem + kOffAbort);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+    const int i0 = p.cta_indptr_tensor[blockIdx.x], i1 = p.cta_indptr_tensor[blockIdx.x + 1];
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar(kQFull), 128);
+        mbar_init(bar(kPFull), 128);
+        mbar_init(bar(kPvDone), 1);
+        mbar_init(bar(kOFree), 128);
+        mbar_init(bar(kSFull0), 1);
+        mbar_init(bar(kSFull1), 1);
+        for (int s = 0; s < kKS; ++s) { mbar_init(bar(kKFull0 + s), 1); mbar_init(bar(kKEmpty0 + s), 1); }
+        for (int s = 0; s < kVS; ++s) { mbar_init(bar(kVFull0 + s), 1); mbar_init(bar(kVEmpty0 + s), 1); }
+        mbar_init(bar(kMmaDrain), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(sbase + kOffTmemPtr), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_ptr;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ producer warp
+        auto load_pages = [&](const TItem& it, int first_page) {
+            const int npg = (it.kv_end - it.kv0 + kPage - 1) / kPage;
+            const int idx = first_page + lane;
+            return idx < npg ? __ldg(p.page_indices + it.page0 + idx) : 0;
+        };
+        constexpr int kPagesPerTile = kTile / kPage;          // 8
+        constexpr int kGroupTiles = 32 / kPagesPerTile;       // 4
+        bool ok = true;
+        int n = 0;                                             // tiles issued so far
+        TItem cur = load_titem(p, i0, i1), nxt = load_titem(p, i0 + 1, i1);
+        int pages_cur = cur.kv_end > 0 ? load_pages(cur, 0) : 0;
+        for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
+            const TItem after = load_titem(p, ii + 2, i1);
+            const int ntiles = (cur.kv_end - cur.kv0 + kTile - 1) / kTile;
+            for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
+                int pages_nxt = 0;
+                if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
+                else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
+                const int t1 = min(t0 + kGroupTiles, ntiles);
+                for (int t = t0; t < t1 && ok; ++t, ++n) {
+                    const int rows = min(kTile, cur.kv_end - (cur.kv0 + t * kTile));
+                    const int npages = (rows + kPage - 1) / kPage;
+                    const int page = __shfl_sync(0xffffffffu, pages_cur, (t - t0) * kPagesPerTile + (lane >> 1 & 7));
+                    const int half = lane & 1;
+                    // K
+                    {
+                        const int s = n % kKS;
+                        ok = mbar_wait_warp(bar(kKEmpty0 + s), ((uint32_t)(n / kKS) & 1u) ^ 1u, abort_flag, p.status, 11);
+                        if (!ok) break;
+                        if (lane == 0) mbar_arrive_expect_tx(bar(kKFull0 + s), (uint32_t)npages * 2 * kBoxBytes);
+                        __syncwarp();
+                        if (lane < 2 * npages) {
+                            const int y = (int)((((int64_t)page * 2 + 0) * Hkv + cur.kv_head) * kPage);
+                            tma_load_2d(sbase + kOffK + s * kTileBytes + half * kHalfBytes + (lane >> 1) * kBoxBytes,
+                                        &kv_map, half * 64, y, bar(kKFull0 + s));
+                        }
+                    }
+                    // V
+                    {
+                        const int s = n % kVS;
+                        ok = mbar_wait_warp(bar(kVEmpty0 + s), ((uint32_t)(n / kVS) & 1u) ^ 1u, abort_flag, p.status, 12);
+                        if (!ok) break;
+                        if (lane == 0) mbar_arrive_expect_tx(bar(kVFull0 + s), (uint32_t)npages * 2 * kBoxBytes);
+                        __syncwarp();
+                        if (lane < 2 * npages) {
+                            const int y = (int)((((int64_t)page * 2 + 1) * Hkv + cur.kv_head) * kPage);
+                            tma_load_2d(sbase + kOffV + s * kTileBytes + half * kHalfBytes + (lane >> 1) * kBoxBytes,
+                                        &kv_map, half * 64, y, bar(kVFull0 + s));
+                        }
+                    }
+                }
+                pages_cur = pages_nxt;
+            }
+            cur = nxt;
+            nxt = after;
+        }
+        if (!ok) {
+            // aborted: let the loads already issued land before shared memory goes away
+            const long long t0 = clock64();
+            for (int k = max(0, n - kKS); k < n; ++k) {
+                while (!mbar_try_wait(bar(kKFull0 + k % kKS), (uint32_t)(k / kKS) & 1u) && clock64() - t0 < kWaitCycles) {}
+                while (!mbar_try_wait(bar(kVFull0 + k % kVS), (uint32_t)(k / kVS) & 1u) && clock64() - t0 < kWaitCycles) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            int gt = 0;          // tiles issued so far (all items): ring and S-buffer position
+            int item_no = 0;
+            const uint32_t idesc_pv = instr_desc(128, 1);
+            for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
+                const TItem it = load_titem(p, ii, i1);
+                const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
+                auto npages_of = [&](int j) {
+                    return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
+                };
+                auto issue_qk = [&](int j) {
+                    const int g = gt + j;
+                    const int s = g % kKS;
+                    if (!mbar_wait(bar(kKFull0 + s), (uint32_t)(g / kKS) & 1u, abort_flag, p.status, 21)) return false;
+                    tc_fence_after();
+                    const uint32_t idesc = instr_desc(16u * (uint32_t)npages_of(j), 0);
+                    const uint32_t d = tmem + kColS + 128u * (uint32_t)(g & 1);
+#pragma unroll
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                        mma_f16(d, smem_desc(sbase + kOffQ + off, 16, 1024),
+                                smem_desc(sbase + kOffK + s * kTileBytes + off, 16, 1024), idesc, ks > 0);
+                    }
+                    mma_commit(bar(kKEmpty0 + s));
+                    mma_commit(bar(kSFull0 + (g & 1)));
+                    return true;
+                };
+                ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
+                if (!ok) break;
+                tc_fence_after();
+                ok = issue_qk(0);
+                for (int j = 0; j < ntiles && ok; ++j) {
+                    if (j + 1 < ntiles) { ok = issue_qk(j + 1); if (!ok) break; }
+                    const int g = gt + j;
+                    const int s = g % kVS;
+                    ok = mbar_wait(bar(kPFull), (uint32_t)g & 1u, abort_flag, p.status, 23) &&
+                         mbar_wait(bar(kVFull0 + s), (uint32_t)(g / kVS) & 1u, abort_flag, p.status, 24);
+                    if (ok && j == 0 && item_no > 0)
+                        ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int npg = npages_of(j);
+                    for (int ks = 0; ks < npg; ++ks) {
+                        const uint32_t poff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                        mma_f16(tmem + kColO, smem_desc(sbase + kOffP + poff, 16, 1024),
+                                smem_desc(sbase + kOffV + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
+                                idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    mma_commit(bar(kVEmpty0 + s));
+                    mma_commit(bar(kPvDone));
+                }
+                gt += ntiles;
+            }
+            // make sure nothing is still running on the tensor core before tensor memory is released
+            mma_commit(bar(kMmaDrain));
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar(kMmaDrain), 0) && clock64() - t0 < kWaitCycles) {}
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ softmax / epilogue warps
+        const int m = threadIdx.x;                 // query row of the tile = tensor-memory lane
+        const int t = m / G, g = m % G;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const float qscale = p.sm_scale * kLog2e;
+        int gt = 0;
+        int item_no = 0;
+        bool ok = true;
+        for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
+            const TItem it = load_titem(p, ii, i1);
+            const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
+            const bool row_valid = t < it.ntok;
+            // ---- stage Q: row m, 16 chunks of 16 bytes, 128-byte swizzle inside each 64-value half
+            {
+                const uint4* src = reinterpret_cast<const uint4*>(
+                    q + ((size_t)(it.q_row0 + t) * Hq + (size_t)it.kv_head * G + g) * kD);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 w = row_valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(smem + kOffQ + (c >> 3) * kHalfBytes + m * 128 + (((c & 7) ^ (m & 7)) << 4)) = w;
+                }
+                fence_async_smem();
+                mbar_arrive(bar(kQFull));
+            }
+            const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
+            float m_ref = -INFINITY, l_sum = 0.f;
+            for (int j = 0; j < ntiles && ok; ++j) {
+                const int gidx = gt + j;
+                const int base = it.kv0 + j * kTile;
+                const int vis = max(0, min(kTile, lim_row - base));     // visible columns of this row
+                ok = mbar_wait_warp(bar(kSFull0 + (gidx & 1)), (uint32_t)(gidx >> 1) & 1u, abort_flag, p.status, 31);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t s_addr = lane_addr + kColS + 128u * (uint32_t)(gidx & 1);
+                const bool full_tile = __all_sync(0xffffffffu, vis == kTile);
+                // pass 1: row maximum
+                float tmax = -INFINITY;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(s_addr + 32u * c, r);
+                    tmem_wait_ld();
+                    if (full_tile) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            tmax = fmaxf(tmax, c * 32 + e < vis ? __uint_as_float(r[e]) : -INFINITY);
+                    }
+                }
+                tmax *= qscale;     // qscale > 0, so the maximum commutes with the scaling
+                // the previous tile's P.V must be done before P is overwritten or O is rescaled
+                if (j > 0) {
+                    ok = mbar_wait_warp(bar(kPvDone), (uint32_t)(gidx - 1) & 1u, abort_flag, p.status, 32);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                const bool grow = tmax > m_ref + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_new = fmaxf(m_ref, tmax);
+                    const float scale = m_new == -INFINITY ? 1.f : fast_exp2(m_ref - m_new);
+                    m_ref = m_new;
+                    l_sum *= scale;
+                    if (j > 0) {
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t r[32];
+                            tmem_ld32(lane_addr + kColO + 32u * c, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * scale);
+                            tmem_st32(lane_addr + kColO + 32u * c, r);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                // pass 2: P = exp2(S * scale - m_ref) as bf16 into shared memory (A operand of P.V)
+                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(s_addr + 32u * c, r);
+                    tmem_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), qscale, -m_use));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), qscale, -m_use));
+                        if (!full_tile) {
+                            if (c * 32 + e >= vis) p0 = 0.f;
+                            if (c * 32 + e + 1 >= vis) p1 = 0.f;
+                        }
+                        l_sum += p0 + p1;
+                        pk[e >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    // columns [32c, 32c+32) = 4 chunks of 8 keys; key half c >> 1, chunks (c & 1) * 4 ..
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int cc = (c & 1) * 4 + k;
+                        *reinterpret_cast<uint4*>(smem + kOffP + (c >> 1) * kHalfBytes + m * 128 + ((cc ^ (m & 7)) << 4)) =
+                            make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+                    }
+                }
+                // last tile: rows of V behind the last key may hold arbitrary bit patterns; zero them so
+                // that 0 * garbage cannot reach O
+                const int rows = min(kTile, it.kv_end - base);
+                if (warp == 0 && (rows & (kPage - 1)) != 0) {
+                    const int sv = gidx % kVS;
+                    ok = mbar_wait_warp(bar(kVFull0 + sv), (uint32_t)(gidx / kVS) & 1u, abort_flag, p.status, 33);
+                    const int r0 = rows, r1 = (rows + kPage - 1) & ~(kPage - 1);
+                    for (int idx = lane; ok && idx < (r1 - r0) * 16; idx += 32) {
+                        const int rr = r0 + idx / 16, ch = idx % 16;
+                        *reinterpret_cast<uint4*>(smem + kOffV + sv * kTileBytes + (ch >> 3) * kHalfBytes + rr * 128 + ((ch & 7) << 4)) =
+                            make_uint4(0, 0, 0, 0);
+                    }
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(bar(kPFull));
+            }
+            if (!ok) break;
+            // ---- epilogue
+            ok = mbar_wait_warp(bar(kPvDone), (uint32_t)(gt + ntiles - 1) & 1u, abort_flag, p.status, 34);
+            if (!ok) break;
+            tc_fence_after();
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const float lse2 = l_sum > 0.f ? m_ref + log2f(l_sum) : -INFINITY;
+            const size_t hq = (size_t)it.kv_head * G + g;
+            const size_t prow = it.partial_base < 0 ? 0 : (size_t)it.partial_base + (size_t)it.chunk * it.ntok + t;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(lane_addr + kColO + 32u * c, r);
+                tmem_wait_ld();
+                if (row_valid) {
+                    if (it.partial_base < 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(it.q_row0 + t) * Hq + hq) * kD + c * 32);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            dst[k] = make_uint4(
+                                pack_bf16x2(__uint_as_float(r[8 * k]) * inv, __uint_as_float(r[8 * k + 1]) * inv),
+                                pack_bf16x2(__uint_as_float(r[8 * k + 2]) * inv, __uint_as_float(r[8 * k + 3]) * inv),
+                                pack_bf16x2(__uint_as_float(r[8 * k + 4]) * inv, __uint_as_float(r[8 * k + 5]) * inv),
+                                pack_bf16x2(__uint_as_float(r[8 * k + 6]) * inv, __uint_as_float(r[8 * k + 7]) * inv));
+                    } else {
+                        float4* dst = reinterpret_cast<float4*>(p.partial_o + (prow * G + g) * kD + c * 32);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            dst[k] = l_sum > 0.f
+                                         ? make_float4(__uint_as_float(r[4 * k]) * inv, __uint_as_float(r[4 * k + 1]) * inv,
+                                                       __uint_as_float(r[4 * k + 2]) * inv, __uint_as_float(r[4 * k + 3]) * inv)
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+            }
+            if (row_valid) {
+                if (it.partial_base < 0) {
+                    if (lse != nullptr) lse[(size_t)(it.q_row0 + t) * Hq + hq] = lse2 * kLn2;
+                } else {
+                    p.partial_lse[prow * G + g] = lse2;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(kOFree));
+            gt += ntiles;
+        }
+    }
+
+    // common exit: every role gets here, then the allocating warp releases tensor memory
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)sym;
+    }
+    return fn;
+}
+
+template <int G>
+static cudaError_t launch_g(const DevPlan& p, const CUtensorMap& map, const void* q, void* out, float* lse,
+                            cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attn_append_tc_kernel<G><<<p.num_ctas_tensor, kThreads, kSmemBytes, stream>>>(
+        p, map, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+
+bool tensor_path_compiled(int head_dim) { return head_dim == tc::kD; }
+
+cudaError_t launch_attn_append_tc(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
+                                  cudaStream_t stream) {
+    if (p.num_items_tensor == 0) return cudaSuccess;
+    if (p.head_dim != tc::kD) return cudaErrorInvalidValue;
+    tc::EncodeTiledFn encode = tc::encode_fn();
+    if (encode == nullptr) return cudaErrorNotSupported;
+    // the pool seen as a matrix of [num_pages * 2 * Hkv * 16 rows][128 values]
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)tc::kD, (cuuint64_t)p.num_pages * 2ull * (cuuint64_t)p.num_kv_heads * kPage};
+    const cuuint64_t strides[1] = {(cuuint64_t)tc::kD * 2};
+    const cuuint32_t box[2] = {64, kPage};
+    const cuuint32_t estr[2] = {1, 1};
+    if (dims[1] == 0 || dims[1] > 0x7fffffffull) return cudaErrorInvalidValue;
+    const CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kv_pool), dims, strides,
+                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    switch (p.group) {
+        case 1: return tc::launch_g<1>(p, map, q, out, lse, stream);
+        case 2: return tc::launch_g<2>(p, map, q, out, lse, stream);
+        case 4: return tc::launch_g<4>(p, map, q, out, lse, stream);
+        case 8: return tc::launch_g<8>(p, map, q, out, lse, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace asynclm
