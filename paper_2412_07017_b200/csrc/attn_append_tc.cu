@@ -6,18 +6,23 @@
 // rows against the same K/V, which is a dense contraction: rows are packed 128 to a tile
 // (row m = token m / G, head m % G) and S = Q K^T and O += P V run on the tensor cores.
 //
-// One persistent CTA per SM, six warps:
-//   warps 0-3  one thread per query row: Q staging, softmax on S read from tensor memory, P written
-//              to shared memory as bf16, lazy rescaling of O, epilogue
-//   warp 4     producer: tiled TMA loads of K/V pages (16 tokens x 64 values per box, 128-byte
-//              swizzle) into two-stage rings
-//   warp 5     one thread issues the MMAs; the warp owns the tensor-memory allocation
-// S is double buffered in tensor memory so that Q K^T of the next tile runs under the softmax of the
-// current one.  All hand-offs are mbarriers with bounded waits; a wait that runs out sets the plan's
-// status word and a CTA-wide abort flag, every role falls through to the common exit, and the
-// tensor memory is released there.
-#include <cuda.h>
-
+// One persistent CTA per SM, ten warps:
+//   warps 0-3, 4-7  two softmax groups, one thread per query row each.  Group b takes the KV tiles
+//                   j = b, b+2, ... of an item and owns S[b], P[b] and O[b]: softmax on S read from
+//                   tensor memory, P written to shared memory as bf16, lazy rescaling of O[b].  The
+//                   two running (max, sum, O) states are merged in the epilogue like two KV splits.
+//   warps 8, 10     producers of the K ring and of the V ring: 16-byte cp.async copies (fully coalesced,
+//                   two 256-byte rows per warp instruction) that write the 128-byte-swizzled operand
+//                   layout directly and complete on the stage's mbarrier; rows behind the last key are
+//                   zero-filled.  (Tiled TMA would need 32 boxes of 2 KiB per 128-key tile, and the
+//                   measured cost of about 90 cycles per small bulk/TMA copy made that the bottleneck.)
+//                   The two rings run independently so that a K tile never queues behind a V stage
+//                   that is still waiting for its P V to finish.
+//   warp 9          one thread issues the MMAs; the warp owns the tensor-memory allocation
+// While one group runs the softmax of tile j the tensor core computes Q K^T of tile j+1 and P V of
+// tile j-1 for the other group.  All hand-offs are mbarriers with bounded waits; a wait that runs
+// out sets the plan's status word and a CTA-wide abort flag, every role falls through to the common
+// exit, and the tensor memory is released there.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -25,31 +30,33 @@ namespace asynclm {
 
 namespace tc {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 352;
+constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10;
 constexpr int kD = 128;
 constexpr int kTile = 128;                       // keys per KV tile and query rows per tile
 constexpr int kKS = 2, kVS = 2;                  // ring depths
 constexpr uint32_t kHalfBytes = 128 * 128;       // one 64-value half of a 128-row tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;  // 32 KiB
-constexpr uint32_t kBoxBytes = 16 * 128;         // one TMA box: 16 tokens x 64 values
 constexpr float kRescaleThreshold = 8.f;
 constexpr long long kWaitCycles = 2000000000ll;
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffP = kOffQ + kTileBytes;
-constexpr uint32_t kOffK = kOffP + kTileBytes;
+constexpr uint32_t kOffP = kOffQ + kTileBytes;          // P[0], P[1]
+constexpr uint32_t kOffK = kOffP + 2 * kTileBytes;
 constexpr uint32_t kOffV = kOffK + kKS * kTileBytes;
 constexpr uint32_t kOffBar = kOffV + kVS * kTileBytes;
-enum Bar { kQFull = 0, kPFull, kPvDone, kOFree, kSFull0, kSFull1, kKFull0, kKEmpty0 = kKFull0 + kKS,
-           kVFull0 = kKEmpty0 + kKS, kVEmpty0 = kVFull0 + kVS, kMmaDrain = kVEmpty0 + kVS, kNumBars };
+enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPFull1, kPvDone0, kPvDone1, kSFull0, kSFull1, kKFull0,
+           kKEmpty0 = kKFull0 + kKS, kVFull0 = kKEmpty0 + kKS, kVEmpty0 = kVFull0 + kVS,
+           kMmaDrain = kVEmpty0 + kVS, kNumBars };
 constexpr uint32_t kOffTmemPtr = kOffBar + 8 * kNumBars;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
 constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
+static_assert(kSmemBytes <= 232448, "shared memory budget");
 
 // tensor memory columns
-constexpr uint32_t kColS = 0;      // two S buffers of 128 columns
-constexpr uint32_t kColO = 256;    // O accumulator, 128 columns
+constexpr uint32_t kColS = 0;      // S[0], S[1]: 128 columns each
+constexpr uint32_t kColO = 256;    // O[0], O[1]: 128 columns each
 constexpr uint32_t kTmemCols = 512;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -95,12 +102,13 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 2-D tiled TMA load (no multicast): box (64 values, 16 rows) at (x, y) of the pool viewed as
-// [rows][128 values].
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+// Arrive on the mbarrier once all cp.async copies issued so far by this thread have landed.
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1.
@@ -177,8 +185,8 @@ __device__ __forceinline__ TItem load_titem(const DevPlan& p, int ii, int i1) {
 
 template <int G>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
-                      const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out,
+attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
+                      const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out,
                       float* __restrict__ lse) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -194,20 +202,22 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
     const int i0 = p.cta_indptr_tensor[blockIdx.x], i1 = p.cta_indptr_tensor[blockIdx.x + 1];
 
     if (threadIdx.x == 0) {
-        mbar_init(bar(kQFull), 128);
-        mbar_init(bar(kPFull), 128);
-        mbar_init(bar(kPvDone), 1);
-        mbar_init(bar(kOFree), 128);
-        mbar_init(bar(kSFull0), 1);
-        mbar_init(bar(kSFull1), 1);
-        for (int s = 0; s < kKS; ++s) { mbar_init(bar(kKFull0 + s), 1); mbar_init(bar(kKEmpty0 + s), 1); }
-        for (int s = 0; s < kVS; ++s) { mbar_init(bar(kVFull0 + s), 1); mbar_init(bar(kVEmpty0 + s), 1); }
+        mbar_init(bar(kQFull), 256);
+        mbar_init(bar(kStats), 256);
+        mbar_init(bar(kOFree), 256);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(kPFull0 + b), 128);
+            mbar_init(bar(kPvDone0 + b), 1);
+            mbar_init(bar(kSFull0 + b), 1);
+        }
+        for (int s = 0; s < kKS; ++s) { mbar_init(bar(kKFull0 + s), 32); mbar_init(bar(kKEmpty0 + s), 1); }
+        for (int s = 0; s < kVS; ++s) { mbar_init(bar(kVFull0 + s), 32); mbar_init(bar(kVEmpty0 + s), 1); }
         mbar_init(bar(kMmaDrain), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(sbase + kOffTmemPtr), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -217,8 +227,12 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
     tc_fence_after();
     const uint32_t tmem = *tmem_ptr;
 
-    if (warp == 4) {
-        // ------------------------------------------------------------------ producer warp
+    if (warp == kProducerWarpK || warp == kProducerWarpV) {
+        // ------------------------------------------------------------------ producer warps
+        const int which = warp == kProducerWarpV ? 1 : 0;       // 0: K ring, 1: V ring
+        const int stages = which ? kVS : kKS;
+        const int full0 = which ? kVFull0 : kKFull0, empty0 = which ? kVEmpty0 : kKEmpty0;
+        const uint32_t ring = sbase + (which ? kOffV : kOffK);
         auto load_pages = [&](const TItem& it, int first_page) {
             const int npg = (it.kv_end - it.kv0 + kPage - 1) / kPage;
             const int idx = first_page + lane;
@@ -241,34 +255,26 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
                 for (int t = t0; t < t1 && ok; ++t, ++n) {
                     const int rows = min(kTile, cur.kv_end - (cur.kv0 + t * kTile));
                     const int npages = (rows + kPage - 1) / kPage;
-                    const int page = __shfl_sync(0xffffffffu, pages_cur, (t - t0) * kPagesPerTile + (lane >> 1 & 7));
-                    const int half = lane & 1;
-                    // K
-                    {
-                        const int s = n % kKS;
-                        ok = mbar_wait_warp(bar(kKEmpty0 + s), ((uint32_t)(n / kKS) & 1u) ^ 1u, abort_flag, p.status, 11);
-                        if (!ok) break;
-                        if (lane == 0) mbar_arrive_expect_tx(bar(kKFull0 + s), (uint32_t)npages * 2 * kBoxBytes);
-                        __syncwarp();
-                        if (lane < 2 * npages) {
-                            const int y = (int)((((int64_t)page * 2 + 0) * Hkv + cur.kv_head) * kPage);
-                            tma_load_2d(sbase + kOffK + s * kTileBytes + half * kHalfBytes + (lane >> 1) * kBoxBytes,
-                                        &kv_map, half * 64, y, bar(kKFull0 + s));
+                    const int s = n % stages;
+                    ok = mbar_wait_warp(bar(empty0 + s), ((uint32_t)(n / stages) & 1u) ^ 1u, abort_flag, p.status, 11 + which);
+                    if (!ok) break;
+                    // lane -> 16-byte chunk c of row 2*rr + (lane >> 4) of each page: a warp instruction
+                    // moves two whole 256-byte rows
+                    const int c = lane & 15;
+                    const uint32_t dst_half = ring + s * kTileBytes + (uint32_t)(c >> 3) * kHalfBytes;
+                    for (int pg = 0; pg < npages; ++pg) {
+                        const int64_t page = __shfl_sync(0xffffffffu, pages_cur, (t - t0) * kPagesPerTile + pg);
+                        const uint8_t* src_page = reinterpret_cast<const uint8_t*>(
+                            pool + pool_row_offset(page, which, cur.kv_head, 0, Hkv, kD));
+#pragma unroll
+                        for (int rr = 0; rr < kPage / 2; ++rr) {
+                            const int slot = rr * 2 + (lane >> 4);
+                            const int row = pg * kPage + slot;
+                            cp_async16(dst_half + (uint32_t)row * 128u + (uint32_t)(((c & 7) ^ (row & 7)) << 4),
+                                       src_page + slot * (kD * 2) + c * 16, row < rows ? 16u : 0u);
                         }
                     }
-                    // V
-                    {
-                        const int s = n % kVS;
-                        ok = mbar_wait_warp(bar(kVEmpty0 + s), ((uint32_t)(n / kVS) & 1u) ^ 1u, abort_flag, p.status, 12);
-                        if (!ok) break;
-                        if (lane == 0) mbar_arrive_expect_tx(bar(kVFull0 + s), (uint32_t)npages * 2 * kBoxBytes);
-                        __syncwarp();
-                        if (lane < 2 * npages) {
-                            const int y = (int)((((int64_t)page * 2 + 1) * Hkv + cur.kv_head) * kPage);
-                            tma_load_2d(sbase + kOffV + s * kTileBytes + half * kHalfBytes + (lane >> 1) * kBoxBytes,
-                                        &kv_map, half * 64, y, bar(kVFull0 + s));
-                        }
-                    }
+                    cp_async_arrive(bar(full0 + s));
                 }
                 pages_cur = pages_nxt;
             }
@@ -278,16 +284,15 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
         if (!ok) {
             // aborted: let the loads already issued land before shared memory goes away
             const long long t0 = clock64();
-            for (int k = max(0, n - kKS); k < n; ++k) {
-                while (!mbar_try_wait(bar(kKFull0 + k % kKS), (uint32_t)(k / kKS) & 1u) && clock64() - t0 < kWaitCycles) {}
-                while (!mbar_try_wait(bar(kVFull0 + k % kVS), (uint32_t)(k / kVS) & 1u) && clock64() - t0 < kWaitCycles) {}
-            }
+            for (int k = max(0, n - stages); k < n; ++k)
+                while (!mbar_try_wait(bar(full0 + k % stages), (uint32_t)(k / stages) & 1u) && clock64() - t0 < kWaitCycles) {}
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             bool ok = true;
-            int gt = 0;          // tiles issued so far (all items): ring and S-buffer position
+            int gt = 0;               // KV tiles issued so far (all items): ring position
+            int cnt[2] = {0, 0};      // tiles handed to each softmax group so far: S/P/PvDone phase
             int item_no = 0;
             const uint32_t idesc_pv = instr_desc(128, 1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
@@ -296,13 +301,14 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
                 auto npages_of = [&](int j) {
                     return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
                 };
+                // S[b] <- Q K_j^T for tile j of the item (b = j & 1); cnt[b] counts tiles of group b
                 auto issue_qk = [&](int j) {
-                    const int g = gt + j;
+                    const int g = gt + j, b = j & 1;
                     const int s = g % kKS;
                     if (!mbar_wait(bar(kKFull0 + s), (uint32_t)(g / kKS) & 1u, abort_flag, p.status, 21)) return false;
                     tc_fence_after();
                     const uint32_t idesc = instr_desc(16u * (uint32_t)npages_of(j), 0);
-                    const uint32_t d = tmem + kColS + 128u * (uint32_t)(g & 1);
+                    const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
@@ -310,18 +316,18 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
                                 smem_desc(sbase + kOffK + s * kTileBytes + off, 16, 1024), idesc, ks > 0);
                     }
                     mma_commit(bar(kKEmpty0 + s));
-                    mma_commit(bar(kSFull0 + (g & 1)));
+                    mma_commit(bar(kSFull0 + b));
                     return true;
                 };
                 ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
                 if (!ok) break;
                 tc_fence_after();
                 ok = issue_qk(0);
+                if (ok && ntiles > 1) ok = issue_qk(1);
                 for (int j = 0; j < ntiles && ok; ++j) {
-                    if (j + 1 < ntiles) { ok = issue_qk(j + 1); if (!ok) break; }
-                    const int g = gt + j;
+                    const int g = gt + j, b = j & 1;
                     const int s = g % kVS;
-                    ok = mbar_wait(bar(kPFull), (uint32_t)g & 1u, abort_flag, p.status, 23) &&
+                    ok = mbar_wait(bar(kPFull0 + b), (uint32_t)(cnt[b] + (j >> 1)) & 1u, abort_flag, p.status, 23) &&
                          mbar_wait(bar(kVFull0 + s), (uint32_t)(g / kVS) & 1u, abort_flag, p.status, 24);
                     if (ok && j == 0 && item_no > 0)
                         ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
@@ -330,14 +336,18 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
                     const int npg = npages_of(j);
                     for (int ks = 0; ks < npg; ++ks) {
                         const uint32_t poff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        mma_f16(tmem + kColO, smem_desc(sbase + kOffP + poff, 16, 1024),
+                        mma_f16(tmem + kColO + 128u * (uint32_t)b,
+                                smem_desc(sbase + kOffP + b * kTileBytes + poff, 16, 1024),
                                 smem_desc(sbase + kOffV + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
-                                idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                                idesc_pv, (j > 1 || ks > 0) ? 1u : 0u);
                     }
                     mma_commit(bar(kVEmpty0 + s));
-                    mma_commit(bar(kPvDone));
+                    mma_commit(bar(kPvDone0 + b));
+                    if (j + 2 < ntiles) ok = issue_qk(j + 2);
                 }
                 gt += ntiles;
+                cnt[0] += (ntiles + 1) >> 1;
+                cnt[1] += ntiles >> 1;
             }
             // make sure nothing is still running on the tensor core before tensor memory is released
             mma_commit(bar(kMmaDrain));
@@ -346,163 +356,189 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ softmax / epilogue warps
-        const int m = threadIdx.x;                 // query row of the tile = tensor-memory lane
+        // ------------------------------------------------------------------ softmax / epilogue groups
+        const int b = warp >> 2;                   // softmax group
+        const int m = threadIdx.x & 127;           // query row of the tile = tensor-memory lane
         const int t = m / G, g = m % G;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t s_addr = lane_addr + kColS + 128u * (uint32_t)b;
+        const uint32_t o_addr = lane_addr + kColO + 128u * (uint32_t)b;
+        uint8_t* p_smem = smem + kOffP + b * kTileBytes;
+        // (max, sum) of each group and row for the epilogue live at the start of that group's P buffer:
+        // P[b] is idle from the group's last P.V until the next item's first Q K^T, which cannot be
+        // issued before every thread has read the statistics and staged the next Q.
+        float2* stats0 = reinterpret_cast<float2*>(smem + kOffP);
+        float2* stats1 = reinterpret_cast<float2*>(smem + kOffP + kTileBytes);
         const float qscale = p.sm_scale * kLog2e;
-        int gt = 0;
+        int gt = 0;          // KV tiles before this item (all groups)
+        int cnt = 0;         // tiles this group has processed before this item
         int item_no = 0;
         bool ok = true;
         for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
             const TItem it = load_titem(p, ii, i1);
             const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
             const bool row_valid = t < it.ntok;
-            // ---- stage Q: row m, 16 chunks of 16 bytes, 128-byte swizzle inside each 64-value half
+            // ---- stage Q: row m; group b stages the 8 chunks (16 bytes each) of value half b, with the
+            //      128-byte swizzle the MMA descriptor expects
             {
                 const uint4* src = reinterpret_cast<const uint4*>(
-                    q + ((size_t)(it.q_row0 + t) * Hq + (size_t)it.kv_head * G + g) * kD);
+                    q + ((size_t)(it.q_row0 + t) * Hq + (size_t)it.kv_head * G + g) * kD) + 8 * b;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 0; c < 8; ++c) {
                     const uint4 w = row_valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4*>(smem + kOffQ + (c >> 3) * kHalfBytes + m * 128 + (((c & 7) ^ (m & 7)) << 4)) = w;
+                    *reinterpret_cast<uint4*>(smem + kOffQ + b * kHalfBytes + m * 128 + ((c ^ (m & 7)) << 4)) = w;
                 }
                 fence_async_smem();
                 mbar_arrive(bar(kQFull));
             }
             const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
             float m_ref = -INFINITY, l_sum = 0.f;
-            for (int j = 0; j < ntiles && ok; ++j) {
-                const int gidx = gt + j;
+            int mine = 0;                                                          // tiles of this group so far
+            for (int j = b; j < ntiles && ok; j += 2, ++mine) {
                 const int base = it.kv0 + j * kTile;
                 const int vis = max(0, min(kTile, lim_row - base));     // visible columns of this row
-                ok = mbar_wait_warp(bar(kSFull0 + (gidx & 1)), (uint32_t)(gidx >> 1) & 1u, abort_flag, p.status, 31);
+                ok = mbar_wait_warp(bar(kSFull0 + b), (uint32_t)(cnt + mine) & 1u, abort_flag, p.status, 31);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t s_addr = lane_addr + kColS + 128u * (uint32_t)(gidx & 1);
                 const bool full_tile = __all_sync(0xffffffffu, vis == kTile);
-                // pass 1: row maximum
-                float tmax = -INFINITY;
+                if (mine == 0) {
+                    // first tile of the group: the reference maximum is this tile's row maximum
+                    float tmax = -INFINITY;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(s_addr + 32u * c, r);
-                    tmem_wait_ld();
-                    if (full_tile) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(r[e]));
-                    } else {
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(s_addr + 32u * c, r);
+                        tmem_wait_ld();
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            tmax = fmaxf(tmax, c * 32 + e < vis ? __uint_as_float(r[e]) : -INFINITY);
+                            tmax = fmaxf(tmax, (full_tile || c * 32 + e < vis) ? __uint_as_float(r[e]) : -INFINITY);
                     }
-                }
-                tmax *= qscale;     // qscale > 0, so the maximum commutes with the scaling
-                // the previous tile's P.V must be done before P is overwritten or O is rescaled
-                if (j > 0) {
-                    ok = mbar_wait_warp(bar(kPvDone), (uint32_t)(gidx - 1) & 1u, abort_flag, p.status, 32);
+                    m_ref = tmax * qscale;     // qscale > 0: the maximum commutes with the scaling
+                } else {
+                    // P[b] and O[b] are still in use by the P.V of this group's previous tile
+                    ok = mbar_wait_warp(bar(kPvDone0 + b), (uint32_t)(cnt + mine - 1) & 1u, abort_flag, p.status, 32);
                     if (!ok) break;
                     tc_fence_after();
                 }
-                const bool grow = tmax > m_ref + kRescaleThreshold;
-                if (__any_sync(0xffffffffu, grow)) {
+                // P = exp2(S * scale - m_ref) as bf16 into shared memory (A operand of P.V).  The
+                // reference maximum is only moved when some score exceeds it by the threshold; then O[b]
+                // and the running sum are rescaled and the tile is redone.
+                float l_tile = 0.f;
+#pragma unroll 1
+                for (int attempt = 0; attempt < 2; ++attempt) {
+                    const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+                    float tmax = -INFINITY;
+                    l_tile = 0.f;
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(s_addr + 32u * c, r);
+                        tmem_wait_ld();
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            float s0 = __uint_as_float(r[e]), s1 = __uint_as_float(r[e + 1]);
+                            if (!full_tile) {
+                                if (c * 32 + e >= vis) s0 = -INFINITY;
+                                if (c * 32 + e + 1 >= vis) s1 = -INFINITY;
+                            }
+                            tmax = fmaxf(tmax, fmaxf(s0, s1));
+                            const float p0 = fast_exp2(fmaf(s0, qscale, -m_use));
+                            const float p1 = fast_exp2(fmaf(s1, qscale, -m_use));
+                            l_tile += p0 + p1;
+                            pk[e >> 1] = pack_bf16x2(p0, p1);
+                        }
+                        // columns [32c, 32c+32) = 4 chunks of 8 keys: key half c >> 1, chunks (c & 1) * 4 ..
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int cc = (c & 1) * 4 + k;
+                            *reinterpret_cast<uint4*>(p_smem + (c >> 1) * kHalfBytes + m * 128 + ((cc ^ (m & 7)) << 4)) =
+                                make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+                        }
+                    }
+                    tmax *= qscale;
+                    if (attempt == 1 || !__any_sync(0xffffffffu, tmax > m_ref + kRescaleThreshold)) break;
                     const float m_new = fmaxf(m_ref, tmax);
                     const float scale = m_new == -INFINITY ? 1.f : fast_exp2(m_ref - m_new);
                     m_ref = m_new;
                     l_sum *= scale;
-                    if (j > 0) {
 #pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(lane_addr + kColO + 32u * c, r);
-                            tmem_wait_ld();
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(o_addr + 32u * c, r);
+                        tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * scale);
-                            tmem_st32(lane_addr + kColO + 32u * c, r);
-                        }
-                        tmem_wait_st();
+                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * scale);
+                        tmem_st32(o_addr + 32u * c, r);
                     }
+                    tmem_wait_st();
                 }
-                // pass 2: P = exp2(S * scale - m_ref) as bf16 into shared memory (A operand of P.V)
-                const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(s_addr + 32u * c, r);
-                    tmem_wait_ld();
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(r[e]), qscale, -m_use));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(r[e + 1]), qscale, -m_use));
-                        if (!full_tile) {
-                            if (c * 32 + e >= vis) p0 = 0.f;
-                            if (c * 32 + e + 1 >= vis) p1 = 0.f;
-                        }
-                        l_sum += p0 + p1;
-                        pk[e >> 1] = pack_bf16x2(p0, p1);
-                    }
-                    // columns [32c, 32c+32) = 4 chunks of 8 keys; key half c >> 1, chunks (c & 1) * 4 ..
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int cc = (c & 1) * 4 + k;
-                        *reinterpret_cast<uint4*>(smem + kOffP + (c >> 1) * kHalfBytes + m * 128 + ((cc ^ (m & 7)) << 4)) =
-                            make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
-                    }
-                }
-                // last tile: rows of V behind the last key may hold arbitrary bit patterns; zero them so
-                // that 0 * garbage cannot reach O
-                const int rows = min(kTile, it.kv_end - base);
-                if (warp == 0 && (rows & (kPage - 1)) != 0) {
-                    const int sv = gidx % kVS;
-                    ok = mbar_wait_warp(bar(kVFull0 + sv), (uint32_t)(gidx / kVS) & 1u, abort_flag, p.status, 33);
-                    const int r0 = rows, r1 = (rows + kPage - 1) & ~(kPage - 1);
-                    for (int idx = lane; ok && idx < (r1 - r0) * 16; idx += 32) {
-                        const int rr = r0 + idx / 16, ch = idx % 16;
-                        *reinterpret_cast<uint4*>(smem + kOffV + sv * kTileBytes + (ch >> 3) * kHalfBytes + rr * 128 + ((ch & 7) << 4)) =
-                            make_uint4(0, 0, 0, 0);
-                    }
-                }
+                l_sum += l_tile;
                 fence_async_smem();
                 tc_fence_before();
-                mbar_arrive(bar(kPFull));
+                mbar_arrive(bar(kPFull0 + b));
             }
             if (!ok) break;
-            // ---- epilogue
-            ok = mbar_wait_warp(bar(kPvDone), (uint32_t)(gt + ntiles - 1) & 1u, abort_flag, p.status, 34);
+            // ---- epilogue: merge the two groups' states, group b writes value half b of every row
+            if (mine > 0) {
+                ok = mbar_wait_warp(bar(kPvDone0 + b), (uint32_t)(cnt + mine - 1) & 1u, abort_flag, p.status, 34);
+                if (!ok) break;
+                tc_fence_after();
+            }
+            (b == 0 ? stats0 : stats1)[m] = make_float2(m_ref, l_sum);
+            mbar_arrive(bar(kStats));
+            ok = mbar_wait_warp(bar(kStats), (uint32_t)item_no & 1u, abort_flag, p.status, 35);
             if (!ok) break;
-            tc_fence_after();
-            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-            const float lse2 = l_sum > 0.f ? m_ref + log2f(l_sum) : -INFINITY;
+            const float2 st0 = stats0[m], st1 = stats1[m];
+            const float M = fmaxf(st0.x, st1.x);
+            const float a0 = st0.y > 0.f ? fast_exp2(st0.x - M) : 0.f;
+            const float a1 = st1.y > 0.f ? fast_exp2(st1.x - M) : 0.f;
+            const float L = a0 * st0.y + a1 * st1.y;
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+            const float w0 = a0 * inv, w1 = a1 * inv;
+            const float lse2 = L > 0.f ? M + log2f(L) : -INFINITY;
             const size_t hq = (size_t)it.kv_head * G + g;
             const size_t prow = it.partial_base < 0 ? 0 : (size_t)it.partial_base + (size_t)it.chunk * it.ntok + t;
+            const bool use0 = __any_sync(0xffffffffu, w0 != 0.f), use1 = __any_sync(0xffffffffu, w1 != 0.f);
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(lane_addr + kColO + 32u * c, r);
-                tmem_wait_ld();
+            for (int c = 2 * b; c < 2 * b + 2; ++c) {
+                float acc[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+                if (use0) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_addr + kColO + 32u * c, r);
+                    tmem_wait_ld();
+                    if (w0 != 0.f) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) acc[e] = __uint_as_float(r[e]) * w0;
+                    }
+                }
+                if (use1) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_addr + kColO + 128u + 32u * c, r);
+                    tmem_wait_ld();
+                    if (w1 != 0.f) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) acc[e] = fmaf(__uint_as_float(r[e]), w1, acc[e]);
+                    }
+                }
                 if (row_valid) {
                     if (it.partial_base < 0) {
                         uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(it.q_row0 + t) * Hq + hq) * kD + c * 32);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            dst[k] = make_uint4(
-                                pack_bf16x2(__uint_as_float(r[8 * k]) * inv, __uint_as_float(r[8 * k + 1]) * inv),
-                                pack_bf16x2(__uint_as_float(r[8 * k + 2]) * inv, __uint_as_float(r[8 * k + 3]) * inv),
-                                pack_bf16x2(__uint_as_float(r[8 * k + 4]) * inv, __uint_as_float(r[8 * k + 5]) * inv),
-                                pack_bf16x2(__uint_as_float(r[8 * k + 6]) * inv, __uint_as_float(r[8 * k + 7]) * inv));
+                            dst[k] = make_uint4(pack_bf16x2(acc[8 * k], acc[8 * k + 1]), pack_bf16x2(acc[8 * k + 2], acc[8 * k + 3]),
+                                                pack_bf16x2(acc[8 * k + 4], acc[8 * k + 5]), pack_bf16x2(acc[8 * k + 6], acc[8 * k + 7]));
                     } else {
                         float4* dst = reinterpret_cast<float4*>(p.partial_o + (prow * G + g) * kD + c * 32);
 #pragma unroll
                         for (int k = 0; k < 8; ++k)
-                            dst[k] = l_sum > 0.f
-                                         ? make_float4(__uint_as_float(r[4 * k]) * inv, __uint_as_float(r[4 * k + 1]) * inv,
-                                                       __uint_as_float(r[4 * k + 2]) * inv, __uint_as_float(r[4 * k + 3]) * inv)
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+                            dst[k] = make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
                     }
                 }
             }
-            if (row_valid) {
+            if (row_valid && b == 0) {
                 if (it.partial_base < 0) {
                     if (lse != nullptr) lse[(size_t)(it.q_row0 + t) * Hq + hq] = lse2 * kLn2;
                 } else {
@@ -512,42 +548,27 @@ attn_append_tc_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map,
             tc_fence_before();
             mbar_arrive(bar(kOFree));
             gt += ntiles;
+            cnt += mine;
         }
     }
 
     // common exit: every role gets here, then the allocating warp releases tensor memory
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)sym;
-    }
-    return fn;
-}
-
 template <int G>
-static cudaError_t launch_g(const DevPlan& p, const CUtensorMap& map, const void* q, void* out, float* lse,
+static cudaError_t launch_g(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                             cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     attn_append_tc_kernel<G><<<p.num_ctas_tensor, kThreads, kSmemBytes, stream>>>(
-        p, map, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse);
+        p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse);
     return cudaGetLastError();
 }
 
@@ -559,24 +580,11 @@ cudaError_t launch_attn_append_tc(const DevPlan& p, const void* q, const void* k
                                   cudaStream_t stream) {
     if (p.num_items_tensor == 0) return cudaSuccess;
     if (p.head_dim != tc::kD) return cudaErrorInvalidValue;
-    tc::EncodeTiledFn encode = tc::encode_fn();
-    if (encode == nullptr) return cudaErrorNotSupported;
-    // the pool seen as a matrix of [num_pages * 2 * Hkv * 16 rows][128 values]
-    CUtensorMap map;
-    const cuuint64_t dims[2] = {(cuuint64_t)tc::kD, (cuuint64_t)p.num_pages * 2ull * (cuuint64_t)p.num_kv_heads * kPage};
-    const cuuint64_t strides[1] = {(cuuint64_t)tc::kD * 2};
-    const cuuint32_t box[2] = {64, kPage};
-    const cuuint32_t estr[2] = {1, 1};
-    if (dims[1] == 0 || dims[1] > 0x7fffffffull) return cudaErrorInvalidValue;
-    const CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kv_pool), dims, strides,
-                              box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     switch (p.group) {
-        case 1: return tc::launch_g<1>(p, map, q, out, lse, stream);
-        case 2: return tc::launch_g<2>(p, map, q, out, lse, stream);
-        case 4: return tc::launch_g<4>(p, map, q, out, lse, stream);
-        case 8: return tc::launch_g<8>(p, map, q, out, lse, stream);
+        case 1: return tc::launch_g<1>(p, q, kv_pool, out, lse, stream);
+        case 2: return tc::launch_g<2>(p, q, kv_pool, out, lse, stream);
+        case 4: return tc::launch_g<4>(p, q, kv_pool, out, lse, stream);
+        case 8: return tc::launch_g<8>(p, q, kv_pool, out, lse, stream);
         default: return cudaErrorInvalidValue;
     }
 }

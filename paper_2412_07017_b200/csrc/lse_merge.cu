@@ -11,11 +11,12 @@ __global__ void __launch_bounds__(128)
 lse_merge_kernel(DevPlan p, __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     constexpr int EPL = D / 32;   // output elements per lane
     const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
     const Unit u = p.units[p.split_units[blockIdx.x]];
     const int G = p.group;
-    for (int pair = warp; pair < u.ntok * G; pair += nwarps) {
+    // one warp per (token, head) pair of the unit; blockIdx.y tiles the unit's pairs
+    const int pair = blockIdx.y * nwarps + (threadIdx.x >> 5);
+    if (pair < u.ntok * G) {
         const int t = pair / G, g = pair % G;
         float mx = -INFINITY;
         for (int c = 0; c < u.n_chunks; ++c) {
@@ -50,10 +51,13 @@ lse_merge_kernel(DevPlan p, __nv_bfloat16* __restrict__ out, float* __restrict__
 
 cudaError_t launch_lse_merge(const DevPlan& p, void* out, float* lse, cudaStream_t stream) {
     if (p.num_split_units == 0) return cudaSuccess;
+    // a unit has at most 128 (token, head) pairs (a tensor-core tile); CUDA-core units have G
+    const int max_pairs = p.num_items_tensor > 0 ? 128 : p.group;
+    const dim3 grid(p.num_split_units, (max_pairs + 3) / 4);
     if (p.head_dim == 128)
-        lse_merge_kernel<128><<<p.num_split_units, 128, 0, stream>>>(p, (__nv_bfloat16*)out, lse);
+        lse_merge_kernel<128><<<grid, 128, 0, stream>>>(p, (__nv_bfloat16*)out, lse);
     else
-        lse_merge_kernel<64><<<p.num_split_units, 128, 0, stream>>>(p, (__nv_bfloat16*)out, lse);
+        lse_merge_kernel<64><<<grid, 128, 0, stream>>>(p, (__nv_bfloat16*)out, lse);
     return cudaGetLastError();
 }
 
