@@ -8,10 +8,13 @@
 // Structure: one persistent CTA per SM walks the item list the planner gave it.  A producer warp
 // streams the items' K/V pages (contiguous 16-token blocks) into a shared-memory ring with bulk
 // asynchronous copies that complete on mbarriers, together with a small descriptor and the query
-// rows of each item.  Eight consumer warps each take 8 of a tile's 64 rows: fp32 dot products with
-// packed two-wide FMAs, a transposing shuffle reduction, softmax against a lazily updated reference
-// maximum, and the P.V update; at the end of an item the warps' states are merged through shared
-// memory and written either as final bf16 output or as an fp32 partial for the split-KV merge.
+// rows of each item.  Twelve consumer warps each take 8 rows of a 96-row tile: fp32 dot products
+// with packed two-wide FMAs, a select-free transposing shuffle reduction, softmax against a lazily
+// updated reference maximum, and the P.V update; at the end of an item the warps' states are merged
+// through shared memory and written either as final bf16 output or as an fp32 partial for the
+// split-KV merge.  The path is bound by instruction latency rather than by any one pipe, so the
+// warp count matters: registers are moved from the producer's warpgroup to the consumers
+// (setmaxnreg) to keep twelve of them resident.
 //
 // Every wait is bounded: a wait that runs out sets the plan's device status word and a CTA-wide
 // abort flag, after which all loops fall through and the kernel returns.
@@ -22,10 +25,14 @@ namespace asynclm {
 
 namespace dec {
 
-constexpr int kWarps = 8;                    // consumer warps
-constexpr int kThreads = (kWarps + 1) * 32;  // + 1 producer warp
-constexpr int kTileTok = 64;                 // rows per ring stage (4 pages)
-constexpr int kRowsPerWarp = kTileTok / kWarps;
+constexpr int kWarps = 12;                   // consumer warps (three warpgroups)
+constexpr int kThreads = (kWarps + 4) * 32;  // + the producer's warpgroup (one working warp)
+constexpr int kRowsPerWarp = 8;
+constexpr int kTileTok = kWarps * kRowsPerWarp;   // 96 rows per ring stage (6 pages)
+// Register budget: the CTA is launched with 512 x 128 registers; the producer's warpgroup gives
+// most of its share back and the consumers take it: 384 x 160 + 128 x 24 = 64512 <= 65536.
+constexpr int kRegsConsumer = 160, kRegsProducer = 24;
+static_assert(kWarps * 32 * kRegsConsumer + 128 * kRegsProducer <= 65536, "register split");
 constexpr float kRescaleThreshold = 16.f;    // log2 units a score may exceed the reference max by
 constexpr long long kWaitCycles = 2000000000ll;
 
@@ -123,7 +130,8 @@ struct Geometry {
     static constexpr int TILE_BYTES = (kTileTok / kPage) * PAGE_BYTES;   // K (or V) part of a stage
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
     static constexpr int Q_BYTES = G * D * 2;
-    static constexpr int MERGE_FLOATS = kWarps * G * (D + 2);            // one merge buffer
+    static constexpr int STAT_FLOATS = (kWarps * G + 7) / 8 * 8;         // max (or sum) array, padded to 32 bytes
+    static constexpr int MERGE_FLOATS = 2 * STAT_FLOATS + kWarps * G * D;  // one merge buffer
     // A lane's slot (i, g) holds the partial score of true row i ^ xi and true head g ^ xg, with
     // (xi, xg) = (mask / G, mask % G) and mask as in transpose_reduce.  The finished score of a
     // lane's slot (i, g) sits in slot score_slot(i, g) of the lane whose index differs from its own
@@ -176,7 +184,9 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
 
     const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
 
-    if (warp == kWarps) {
+    if (warp >= kWarps) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
+        if (warp > kWarps) return;      // the other warps of the producer's warpgroup have nothing to do
         // ------------------------------------------------------------------ producer warp
         // The page ids of the next 32 pages (8 tiles) and the descriptors of the next two items are
         // fetched ahead of use, so that no global-load latency sits between two tiles.
@@ -237,7 +247,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
                     }
                     __syncwarp();
                     const int64_t page = __shfl_sync(0xffffffffu, pages_cur,
-                                                     (t - t0) * kPagesPerTile + (lane & (kPagesPerTile - 1)));
+                                                     (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
                     if (lane < npages) {
                         const __nv_bfloat16* src = pool + pool_row_offset(page, 0, cur.kv_head, 0, Hkv, D);
                         const uint32_t dst = smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * Geo::PAGE_BYTES);
@@ -274,6 +284,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     }
 
     // ---------------------------------------------------------------------- consumer warps
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
     const int sub = lane % LPR;
     const int grp = lane / LPR;
     const int my_row = (sub >> 2) * TPW + grp;   // row (within the warp's 8) of this lane's scores
@@ -314,11 +325,12 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             cur_out_row = d.out_row; cur_kv_head = d.kv_head; cur_partial = d.partial_row;
         }
         const int rows = d.rows;
-        const bool active = warp * kRowsPerWarp < rows;
+        const int blk = warp;
+        const bool active = blk * kRowsPerWarp < rows;
         uint4 kw[NR], vw[NR];
         if (active) {
             const uint8_t* ks = stage_base + (size_t)s * Geo::STAGE_BYTES +
-                                (size_t)(warp * kRowsPerWarp) * (D * 2) + lane * 16;
+                                (size_t)(blk * kRowsPerWarp) * (D * 2) + lane * 16;
 #pragma unroll
             for (int i = 0; i < NR; ++i) {
                 kw[i] = *reinterpret_cast<const uint4*>(ks + (size_t)(i ^ xi) * TPW * D * 2);
@@ -329,11 +341,11 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
         if (lane == 0) mbar_arrive(empty0 + 8 * s);
 
         if (active) {
-            const bool tail = rows < (warp + 1) * kRowsPerWarp;
+            const bool tail = rows < (blk + 1) * kRowsPerWarp;
             if (tail) {
 #pragma unroll
                 for (int i = 0; i < NR; ++i)
-                    if (warp * kRowsPerWarp + (i ^ xi) * TPW + grp >= rows) {
+                    if (blk * kRowsPerWarp + (i ^ xi) * TPW + grp >= rows) {
                         kw[i] = make_uint4(0, 0, 0, 0);
                         vw[i] = make_uint4(0, 0, 0, 0);
                     }
@@ -356,7 +368,7 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             float sc[NF];
 #pragma unroll
             for (int f = 0; f < NF; ++f) sc[f] = v[f];
-            if (tail && warp * kRowsPerWarp + my_row >= rows) {
+            if (tail && blk * kRowsPerWarp + my_row >= rows) {
 #pragma unroll
                 for (int f = 0; f < NF; ++f) sc[f] = -INFINITY;
             }
@@ -413,8 +425,8 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
         if (d.flags & kFlagLast) {
             // ---- end of item: merge the warps' states and write the result
             float* mm = merge_base + (size_t)(item_count & 1) * Geo::MERGE_FLOATS;   // [warp][G] max
-            float* ml = mm + kWarps * G;                                          // [warp][G] sum
-            float* mo = ml + kWarps * G;                                          // [warp][G][D]
+            float* ml = mm + Geo::STAT_FLOATS;                                    // [warp][G] sum
+            float* mo = ml + Geo::STAT_FLOATS;                                    // [warp][G][D]
 #pragma unroll
             for (int f = 0; f < NF; ++f) {
                 l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 4);
