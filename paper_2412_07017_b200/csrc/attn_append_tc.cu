@@ -226,6 +226,11 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_ptr;
+    // Launched with programmatic serialization: everything above overlapped the tail of the append
+    // kernel; from here on the pool is read.  Once every CTA has passed this point the CUDA-core
+    // kernel behind this one may start on SMs that become free.
+    pdl_wait();
+    pdl_trigger();
 
     if (warp == kProducerWarpK || warp == kProducerWarpV) {
         // ------------------------------------------------------------------ producer warps
@@ -295,8 +300,10 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             int cnt[2] = {0, 0};      // tiles handed to each softmax group so far: S/P/PvDone phase
             int item_no = 0;
             const uint32_t idesc_pv = instr_desc(128, 1);
+            TItem it_next = load_titem(p, i0, i1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
-                const TItem it = load_titem(p, ii, i1);
+                const TItem it = it_next;
+                it_next = load_titem(p, ii + 1, i1);      // in flight while this item runs
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
                 auto npages_of = [&](int j) {
                     return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
@@ -374,23 +381,30 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
         int cnt = 0;         // tiles this group has processed before this item
         int item_no = 0;
         bool ok = true;
+        // This thread's share of an item's Q: row m, the 8 chunks (16 bytes each) of value half b.  The
+        // next item's descriptor and Q rows are fetched while the current item runs.
+        auto load_q = [&](const TItem& x, uint4 (&w)[8]) {
+            const bool valid = x.kv_end > 0 && t < x.ntok;
+            const uint4* src = reinterpret_cast<const uint4*>(
+                q + ((size_t)(x.q_row0 + t) * Hq + (size_t)x.kv_head * G + g) * kD) + 8 * b;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) w[c] = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+        };
+        TItem it_next = load_titem(p, i0, i1);
+        uint4 q_next[8];
+        load_q(it_next, q_next);
         for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
-            const TItem it = load_titem(p, ii, i1);
+            const TItem it = it_next;
             const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
             const bool row_valid = t < it.ntok;
-            // ---- stage Q: row m; group b stages the 8 chunks (16 bytes each) of value half b, with the
-            //      128-byte swizzle the MMA descriptor expects
-            {
-                const uint4* src = reinterpret_cast<const uint4*>(
-                    q + ((size_t)(it.q_row0 + t) * Hq + (size_t)it.kv_head * G + g) * kD) + 8 * b;
+            // ---- stage Q with the 128-byte swizzle the MMA descriptor expects
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint4 w = row_valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4*>(smem + kOffQ + b * kHalfBytes + m * 128 + ((c ^ (m & 7)) << 4)) = w;
-                }
-                fence_async_smem();
-                mbar_arrive(bar(kQFull));
-            }
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(smem + kOffQ + b * kHalfBytes + m * 128 + ((c ^ (m & 7)) << 4)) = q_next[c];
+            fence_async_smem();
+            mbar_arrive(bar(kQFull));
+            it_next = load_titem(p, ii + 1, i1);
+            load_q(it_next, q_next);
             const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
             float m_ref = -INFINITY, l_sum = 0.f;
             int mine = 0;                                                          // tiles of this group so far
@@ -567,9 +581,8 @@ static cudaError_t launch_g(const DevPlan& p, const void* q, const void* pool, v
     cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    attn_append_tc_kernel<G><<<p.num_ctas_tensor, kThreads, kSmemBytes, stream>>>(
-        p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse);
-    return cudaGetLastError();
+    return launch_pdl(attn_append_tc_kernel<G>, dim3(p.num_ctas_tensor), dim3(kThreads), kSmemBytes, stream, p,
+                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse);
 }
 
 }  // namespace tc

@@ -153,7 +153,7 @@ template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
                    const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out,
-                   float* __restrict__ lse, int S) {
+                   float* __restrict__ lse, int S, int wait_prior) {
     using Geo = Geometry<D, G>;
     constexpr int LPR = Geo::LPR, TPW = Geo::TPW, NR = Geo::NR, NV = Geo::NV, NF = Geo::NF;
     extern __shared__ uint8_t smem_raw[];
@@ -183,6 +183,10 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     __syncthreads();
 
     const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+    // Launched with programmatic serialization.  After the append kernel it must wait for the
+    // appended rows; after the tensor-core kernel (which has itself waited for the append and whose
+    // results it does not read) it only fills the SMs that kernel frees up.
+    if (wait_prior) pdl_wait();
 
     if (warp >= kWarps) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
@@ -507,9 +511,9 @@ static cudaError_t launch_dg(const DevPlan& p, const void* q, const void* pool, 
     cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attn_decode_kernel<D, G><<<p.num_ctas_cuda, kThreads, smem, stream>>>(
-        p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
-    return cudaGetLastError();
+    return launch_pdl(attn_decode_kernel<D, G>, dim3(p.num_ctas_cuda), dim3(kThreads), smem, stream, p,
+                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S,
+                      p.num_items_tensor == 0 ? 1 : 0);
 }
 
 template <int D>

@@ -13,6 +13,7 @@ namespace asynclm {
 __global__ void __launch_bounds__(256)
 kv_append_kernel(DevPlan p, const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                  uint4* __restrict__ pool) {
+    pdl_trigger();   // the attention kernel may start its prologue; it waits for this grid before reading the pool
     const int vpr = p.head_dim / 8;                       // 16-byte vectors per row
     const int64_t total = (int64_t)p.total_q * p.num_kv_heads * 2 * vpr;
     for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;

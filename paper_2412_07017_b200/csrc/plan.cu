@@ -48,11 +48,12 @@ static int default_tensor_min_rows() { return 32; }
 // Sizes of the sections of the packed blob (identical offsets on host and device).
 struct BlobLayout {
     size_t off_q_indptr, off_kv_len, off_page_indptr, off_page_indices, off_row_seq, off_units,
-        off_items, off_cta_cuda, off_cta_tensor, off_split, off_status, blob_bytes;
+        off_items, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
 };
 
 static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64_t n_units,
-                              int64_t n_items, int ctas_cuda, int ctas_tensor, int64_t n_split) {
+                              int64_t n_items, int ctas_cuda, int ctas_tensor, int64_t n_split,
+                              int64_t n_merge_blocks) {
     BlobLayout L{};
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
@@ -67,6 +68,7 @@ static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64
     L.off_cta_cuda = take(sizeof(int32_t) * (size_t)(ctas_cuda + 1));
     L.off_cta_tensor = take(sizeof(int32_t) * (size_t)(ctas_tensor + 1));
     L.off_split = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_split, 1));
+    L.off_merge = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_merge_blocks, 1));
     L.blob_bytes = o;
     return L;
 }
@@ -111,7 +113,8 @@ extern "C" int asynclm_plan_workspace_size(const asynclm_shape* shape,
                            (int64_t)2 * (ctas_cuda + ctas_tensor);
     }
     BlobLayout L = layout_blob(max_batch, max_total_q, max_total_pages, max_units, max_items,
-                               ctas_cuda, ctas_tensor, max_units);
+                               ctas_cuda, ctas_tensor, max_units,
+                               (int64_t)max_total_q * shape->num_q_heads / 4 + max_units);
     *host_bytes = align_up(sizeof(asynclm_plan_s), 256) + L.blob_bytes +
                   align_up(sizeof(int32_t) * (size_t)std::max<int64_t>(max_items, 1), 256);
     *device_bytes = L.blob_bytes + partial_bytes(max_partial_rows, G, shape->head_dim);
@@ -150,17 +153,13 @@ void cut_and_deal(const std::vector<int>& unit_ids, std::vector<UnitBuild>& unit
         int64_t total = 0;
         for (size_t i = first_item; i < items.size(); ++i)
             total += item_overhead_tiles + tiles_of(items[i].kv1 - items[i].kv0);
-        const int64_t quota = (total + n_ctas - 1) / n_ctas;
-        int cta = 0;
-        int64_t load = 0;
+        // contiguous partition: an item goes to the CTA in whose share of the total its midpoint falls
+        int64_t cum = 0;
         for (size_t i = first_item; i < items.size(); ++i) {
             const int64_t c = item_overhead_tiles + tiles_of(items[i].kv1 - items[i].kv0);
-            if (load > 0 && load + c > quota && cta + 1 < n_ctas) {
-                ++cta;
-                load = 0;
-            }
-            load += c;
-            item_cta.push_back(cta);
+            const int64_t cta = std::min<int64_t>(n_ctas - 1, ((2 * cum + c) * n_ctas) / (2 * total));
+            item_cta.push_back((int32_t)cta);
+            cum += c;
         }
     } else {
         int64_t total_tiles = 0;
@@ -333,20 +332,24 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     const int n_items = (int)items.size();
 
     // ---- partial rows ------------------------------------------------------------------------
-    std::vector<int32_t> split_units;
+    std::vector<int32_t> split_units, merge_blocks;   // merge block: 4 (token, head) rows of a split unit
     int64_t partial_rows = 0;
     for (size_t i = 0; i < units.size(); ++i) {
         if (units[i].u.n_chunks > 1) {
             units[i].u.partial_base = (int32_t)partial_rows;
             partial_rows += (int64_t)units[i].u.n_chunks * units[i].u.ntok;
             split_units.push_back((int32_t)i);
+            if (i >= (size_t)(INT32_MAX >> 5)) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
+            for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 5) | (size_t)rb));
             if (partial_rows > INT32_MAX / 2) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
         }
     }
 
+    const int n_split = (int)split_units.size();
+
     // ---- pack ---------------------------------------------------------------------------------
     BlobLayout L = layout_blob(B, T, total_pages, (int64_t)units.size(), n_items, ctas_cuda,
-                               ctas_tensor, (int64_t)split_units.size());
+                               ctas_tensor, (int64_t)n_split, (int64_t)merge_blocks.size());
     const size_t plan_bytes = align_up(sizeof(asynclm_plan_s), 256);
     const size_t item_cta_bytes = align_up(sizeof(int32_t) * (size_t)std::max(n_items, 1), 256);
     const size_t host_need = plan_bytes + L.blob_bytes + item_cta_bytes;
@@ -375,8 +378,9 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     std::memcpy(hb + L.off_cta_cuda, cta_indptr_cuda.data(), sizeof(int32_t) * (size_t)(ctas_cuda + 1));
     std::memcpy(hb + L.off_cta_tensor, cta_indptr_tensor.data(),
                 sizeof(int32_t) * (size_t)(ctas_tensor + 1));
-    if (!split_units.empty())
-        std::memcpy(hb + L.off_split, split_units.data(), sizeof(int32_t) * split_units.size());
+    if (n_split > 0) std::memcpy(hb + L.off_split, split_units.data(), sizeof(int32_t) * split_units.size());
+    if (!merge_blocks.empty())
+        std::memcpy(hb + L.off_merge, merge_blocks.data(), sizeof(int32_t) * merge_blocks.size());
     int32_t* h_item_cta = (int32_t*)(hb + L.blob_bytes);
     if (n_items > 0) std::memcpy(h_item_cta, item_cta.data(), sizeof(int32_t) * (size_t)n_items);
 
@@ -406,6 +410,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     d.cta_indptr_cuda = (const int32_t*)dp(L.off_cta_cuda);
     d.cta_indptr_tensor = (const int32_t*)dp(L.off_cta_tensor);
     d.split_units = (const int32_t*)dp(L.off_split);
+    d.merge_blocks = (const int32_t*)dp(L.off_merge);
     d.partial_o = (float*)dp(L.blob_bytes);
     d.partial_lse = (float*)dp(L.blob_bytes + align_up((size_t)partial_rows * (size_t)G *
                                                            (size_t)shape->head_dim * sizeof(float), 256));
@@ -415,7 +420,8 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     d.num_items = n_items;
     d.num_items_cuda = n_items_cuda;
     d.num_items_tensor = n_items - n_items_cuda;
-    d.num_split_units = (int32_t)split_units.size();
+    d.num_split_units = n_split;
+    d.num_merge_blocks = (int32_t)merge_blocks.size();
     d.num_ctas_cuda = ctas_cuda;
     d.num_ctas_tensor = ctas_tensor;
     d.num_q_heads = shape->num_q_heads;

@@ -13,7 +13,7 @@ constexpr uint64_t kPlanMagic = 0x4153594e434c4d31ull;   // "ASYNCLM1"
 constexpr int kCudaSlotsPerSm = 1;
 // Fixed cost of starting an item, in units of one 128-token KV tile, used when balancing CTAs.
 constexpr int kCudaItemOverheadTiles = 1;
-constexpr int kTensorItemOverheadTiles = 1;
+constexpr int kTensorItemOverheadTiles = 4;   // measured: an item boundary costs the tensor kernel about 4 tiles
 
 // True when the tensor-core attention kernel exists for this head_dim.
 bool tensor_path_compiled(int head_dim);

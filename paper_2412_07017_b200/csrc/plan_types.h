@@ -43,11 +43,13 @@ struct DevPlan {
     const int32_t* cta_indptr_cuda;  // [num_ctas_cuda + 1] into items
     const int32_t* cta_indptr_tensor;// [num_ctas_tensor + 1] into items (absolute indices)
     const int32_t* split_units;      // [num_split_units] unit ids that need a merge
+    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 5) | row block: 4 (token, head) rows each
     float* partial_o;                // [partial_rows][G][d]
     float* partial_lse;              // [partial_rows][G]   (log2 domain)
     int32_t* status;                 // device status word
     int32_t batch, total_q, num_units, num_items, num_items_cuda, num_items_tensor;
     int32_t num_split_units, num_ctas_cuda, num_ctas_tensor;
+    int32_t num_merge_blocks;
     int32_t num_q_heads, num_kv_heads, head_dim, group;
     int64_t num_pages;
     float sm_scale;
