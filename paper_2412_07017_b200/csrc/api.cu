@@ -58,9 +58,7 @@ extern "C" int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, con
     if (!q || !kv_pool || !out || !aligned16(q) || !aligned16(kv_pool) || !aligned16(out))
         return ASYNCLM_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
-    int rc = cuda_status(launch_attn_append_tc(plan->dev, q, kv_pool, out, lse, s));
-    if (rc != ASYNCLM_OK) return rc;
-    rc = cuda_status(launch_attn_decode(plan->dev, q, kv_pool, out, lse, s));
+    int rc = cuda_status(launch_attention(plan->dev, q, kv_pool, out, lse, s));
     if (rc != ASYNCLM_OK) return rc;
     return cuda_status(launch_lse_merge(plan->dev, out, lse, s));
 }

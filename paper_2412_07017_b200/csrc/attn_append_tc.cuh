@@ -23,6 +23,7 @@
 // tile j-1 for the other group.  All hand-offs are mbarriers with bounded waits; a wait that runs
 // out sets the plan's status word and a CTA-wide abort flag, every role falls through to the common
 // exit, and the tensor memory is released there.
+#pragma once
 #include "common.cuh"
 #include "kernels.h"
 
@@ -183,13 +184,18 @@ __device__ __forceinline__ TItem load_titem(const DevPlan& p, int ii, int i1) {
     return r;
 }
 
-template <int G>
-__global__ void __launch_bounds__(kThreads, 1)
-attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
-                      const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out,
-                      float* __restrict__ lse) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+// Register shares of the fused kernel's tensor-core phase (512 threads launched with 128 each):
+// softmax warps 0-7, the producer/MMA warpgroup 8-11, and warps 12-15, which idle in this phase.
+constexpr int kRegsSoftmaxFused = 168, kRegsIssueFused = 80, kRegsIdleFused = 24;
+static_assert(256 * kRegsSoftmaxFused + 128 * kRegsIssueFused + 128 * kRegsIdleFused <= 65536, "register split");
+
+// The whole kernel body.  FUSED: called by all 16 warps of the fused kernel (warps 11-15 only take
+// part in the CTA-wide barriers), with `smem` 1024-byte aligned.
+template <int G, bool FUSED>
+__device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
+                                        const __nv_bfloat16* __restrict__ pool,
+                                        __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+                                        uint8_t* smem) {
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + kOffBar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
@@ -230,9 +236,13 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     // kernel; from here on the pool is read.  Once every CTA has passed this point the CUDA-core
     // kernel behind this one may start on SMs that become free.
     pdl_wait();
-    pdl_trigger();
+    if constexpr (!FUSED) pdl_trigger();
 
-    if (warp == kProducerWarpK || warp == kProducerWarpV) {
+    if (warp >= 12) {
+        if constexpr (FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIdleFused));
+    } else if (warp >= 8) {
+      if constexpr (FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssueFused));
+      if (warp == kProducerWarpK || warp == kProducerWarpV) {
         // ------------------------------------------------------------------ producer warps
         const int which = warp == kProducerWarpV ? 1 : 0;       // 0: K ring, 1: V ring
         const int stages = which ? kVS : kKS;
@@ -362,7 +372,9 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
             while (!mbar_try_wait(bar(kMmaDrain), 0) && clock64() - t0 < kWaitCycles) {}
         }
         __syncwarp();
+      }
     } else {
+        if constexpr (FUSED) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxFused));
         // ------------------------------------------------------------------ softmax / epilogue groups
         const int b = warp >> 2;                   // softmax group
         const int m = threadIdx.x & 127;           // query row of the tile = tensor-memory lane
@@ -575,31 +587,6 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     }
 }
 
-template <int G>
-static cudaError_t launch_g(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
-                            cudaStream_t stream) {
-    cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(attn_append_tc_kernel<G>, dim3(p.num_ctas_tensor), dim3(kThreads), kSmemBytes, stream, p,
-                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse);
-}
-
 }  // namespace tc
-
-bool tensor_path_compiled(int head_dim) { return head_dim == tc::kD; }
-
-cudaError_t launch_attn_append_tc(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
-                                  cudaStream_t stream) {
-    if (p.num_items_tensor == 0) return cudaSuccess;
-    if (p.head_dim != tc::kD) return cudaErrorInvalidValue;
-    switch (p.group) {
-        case 1: return tc::launch_g<1>(p, q, kv_pool, out, lse, stream);
-        case 2: return tc::launch_g<2>(p, q, kv_pool, out, lse, stream);
-        case 4: return tc::launch_g<4>(p, q, kv_pool, out, lse, stream);
-        case 8: return tc::launch_g<8>(p, q, kv_pool, out, lse, stream);
-        default: return cudaErrorInvalidValue;
-    }
-}
 
 }  // namespace asynclm

@@ -18,6 +18,7 @@
 //
 // Every wait is bounded: a wait that runs out sets the plan's device status word and a CTA-wide
 // abort flag, after which all loops fall through and the kernel returns.
+#pragma once
 #include "common.cuh"
 #include "kernels.h"
 
@@ -149,15 +150,15 @@ size_t smem_bytes(int stages) {
            2 * Geo::MERGE_FLOATS * sizeof(float) + 3 * 8 + 16 + 1024;
 }
 
-template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 1)
-attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
-                   const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out,
-                   float* __restrict__ lse, int S, int wait_prior) {
+// The whole kernel body.  FUSED: the CTA has just finished the tensor-core phase of the fused
+// kernel, in which warps 0-7 held 168 registers, warps 8-11 held 80 and warps 12-15 held 24.
+template <int D, int G, bool FUSED>
+__device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
+                                            const __nv_bfloat16* __restrict__ pool,
+                                            __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+                                            int S, uint8_t* smem) {
     using Geo = Geometry<D, G>;
     constexpr int LPR = Geo::LPR, TPW = Geo::TPW, NR = Geo::NR, NV = Geo::NV, NF = Geo::NF;
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* stage_base = smem;
     uint8_t* q_base = stage_base + (size_t)S * Geo::STAGE_BYTES;
     float* merge_base = (float*)(q_base + (size_t)S * Geo::Q_BYTES);
@@ -183,13 +184,9 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     __syncthreads();
 
     const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
-    // Launched with programmatic serialization.  After the append kernel it must wait for the
-    // appended rows; after the tensor-core kernel (which has itself waited for the append and whose
-    // results it does not read) it only fills the SMs that kernel frees up.
-    if (wait_prior) pdl_wait();
 
     if (warp >= kWarps) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
+        if constexpr (!FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
         if (warp > kWarps) return;      // the other warps of the producer's warpgroup have nothing to do
         // ------------------------------------------------------------------ producer warp
         // The page ids of the next 32 pages (8 tiles) and the descriptors of the next two items are
@@ -288,7 +285,12 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     }
 
     // ---------------------------------------------------------------------- consumer warps
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
+    if constexpr (FUSED) {
+        if (warp < 8) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
+        else asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
+    }
     const int sub = lane % LPR;
     const int grp = lane / LPR;
     const int my_row = (sub >> 2) * TPW + grp;   // row (within the warp's 8) of this lane's scores
@@ -502,40 +504,6 @@ attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q,
     }
 }
 
-template <int D, int G>
-static cudaError_t launch_dg(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
-                             cudaStream_t stream) {
-    int S = 8;
-    while (S > 2 && smem_bytes<D, G>(S) > 232448) --S;
-    const size_t smem = smem_bytes<D, G>(S);
-    cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return launch_pdl(attn_decode_kernel<D, G>, dim3(p.num_ctas_cuda), dim3(kThreads), smem, stream, p,
-                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S,
-                      p.num_items_tensor == 0 ? 1 : 0);
-}
-
-template <int D>
-static cudaError_t launch_d(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
-                            cudaStream_t stream) {
-    switch (p.group) {
-        case 1: return launch_dg<D, 1>(p, q, pool, out, lse, stream);
-        case 2: return launch_dg<D, 2>(p, q, pool, out, lse, stream);
-        case 4: return launch_dg<D, 4>(p, q, pool, out, lse, stream);
-        case 8: return launch_dg<D, 8>(p, q, pool, out, lse, stream);
-        default: return cudaErrorInvalidValue;
-    }
-}
-
 }  // namespace dec
-
-cudaError_t launch_attn_decode(const DevPlan& p, const void* q, const void* kv_pool, void* out,
-                               float* lse, cudaStream_t stream) {
-    if (p.num_items_cuda == 0) return cudaSuccess;
-    if (p.head_dim == 128) return dec::launch_d<128>(p, q, kv_pool, out, lse, stream);
-    if (p.head_dim == 64) return dec::launch_d<64>(p, q, kv_pool, out, lse, stream);
-    return cudaErrorInvalidValue;
-}
 
 }  // namespace asynclm

@@ -1,0 +1,143 @@
+// The attention kernels' entry points and launchers.
+//
+// Three kernels are built from two bodies (attn_append_tc.cuh: tensor-core span tiles,
+// attn_decode.cuh: CUDA-core decode rows):
+//   attn_fused_kernel      a persistent CTA first runs its tensor-core items, then its CUDA-core items.
+//                          One launch instead of two: the fixed cost of a launch (about 10 us of
+//                          start-up and tail per kernel at 148 CTAs) is paid once, and a CTA that is
+//                          done with its span tiles early moves on to decode rows at once.
+//   attn_append_tc_kernel  steps that have span tiles only
+//   attn_decode_kernel     steps without span tiles, and head_dim 64
+// All are launched with programmatic stream serialization and wait for the kernel in front of them
+// (normally the KV append) right before they first touch the pool.
+#include "attn_append_tc.cuh"
+#include "attn_decode.cuh"
+
+namespace asynclm {
+
+namespace {
+
+constexpr int kMaxSmem = 232448;
+
+__device__ __forceinline__ uint8_t* aligned_smem(uint8_t* raw) {
+    return (uint8_t*)(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(dec::kThreads, 1)
+attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pool,
+                   __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
+    extern __shared__ uint8_t smem_raw[];
+    pdl_wait();
+    dec::decode_body<D, G, false>(p, q, pool, out, lse, S, aligned_smem(smem_raw));
+}
+
+template <int G>
+__global__ void __launch_bounds__(tc::kThreads, 1)
+attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pool,
+                      __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    extern __shared__ uint8_t smem_raw[];
+    tc::tc_body<G, false>(p, q, pool, out, lse, aligned_smem(smem_raw));
+}
+
+template <int G>
+__global__ void __launch_bounds__(dec::kThreads, 1)
+attn_fused_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pool,
+                  __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = aligned_smem(smem_raw);
+    tc::tc_body<G, true>(p, q, pool, out, lse, smem);
+    __syncthreads();      // tensor memory released, shared memory free for the second phase
+    dec::decode_body<tc::kD, G, true>(p, q, pool, out, lse, S, smem);
+}
+
+template <int D, int G>
+int decode_stages() {
+    int S = 8;
+    while (S > 2 && dec::smem_bytes<D, G>(S) > (size_t)kMaxSmem) --S;
+    return S;
+}
+
+template <int D, int G>
+cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
+                          cudaStream_t stream) {
+    const int S = decode_stages<D, G>();
+    const size_t smem = dec::smem_bytes<D, G>(S);
+    cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(attn_decode_kernel<D, G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p,
+                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
+}
+
+template <int G>
+cudaError_t launch_tensor(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
+                          cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)tc::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(attn_append_tc_kernel<G>, dim3(p.num_ctas_tensor), dim3(tc::kThreads), tc::kSmemBytes, stream,
+                      p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse);
+}
+
+template <int G>
+cudaError_t launch_fused(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
+                         cudaStream_t stream) {
+    const int S = decode_stages<tc::kD, G>();
+    const size_t smem = dec::smem_bytes<tc::kD, G>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD, G>(S) : tc::kSmemBytes;
+    cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(attn_fused_kernel<G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p,
+                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
+}
+
+template <int D>
+cudaError_t launch_decode_d(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
+                            cudaStream_t stream) {
+    switch (p.group) {
+        case 1: return launch_decode<D, 1>(p, q, pool, out, lse, stream);
+        case 2: return launch_decode<D, 2>(p, q, pool, out, lse, stream);
+        case 4: return launch_decode<D, 4>(p, q, pool, out, lse, stream);
+        case 8: return launch_decode<D, 8>(p, q, pool, out, lse, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+bool tensor_path_compiled(int head_dim) { return head_dim == tc::kD; }
+
+cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
+                             cudaStream_t stream) {
+    const bool has_tensor = p.num_items_tensor > 0, has_cuda = p.num_items_cuda > 0;
+    if (has_tensor && p.head_dim != tc::kD) return cudaErrorInvalidValue;
+    if (has_tensor && has_cuda && p.num_ctas_tensor == p.num_ctas_cuda) {
+        switch (p.group) {
+            case 1: return launch_fused<1>(p, q, kv_pool, out, lse, stream);
+            case 2: return launch_fused<2>(p, q, kv_pool, out, lse, stream);
+            case 4: return launch_fused<4>(p, q, kv_pool, out, lse, stream);
+            case 8: return launch_fused<8>(p, q, kv_pool, out, lse, stream);
+            default: return cudaErrorInvalidValue;
+        }
+    }
+    if (has_tensor) {
+        cudaError_t e;
+        switch (p.group) {
+            case 1: e = launch_tensor<1>(p, q, kv_pool, out, lse, stream); break;
+            case 2: e = launch_tensor<2>(p, q, kv_pool, out, lse, stream); break;
+            case 4: e = launch_tensor<4>(p, q, kv_pool, out, lse, stream); break;
+            case 8: e = launch_tensor<8>(p, q, kv_pool, out, lse, stream); break;
+            default: e = cudaErrorInvalidValue;
+        }
+        if (e != cudaSuccess) return e;
+    }
+    if (has_cuda) {
+        // a decode kernel behind a tensor kernel would have to wait for it to finish (pdl_wait), which
+        // is what stream order gives anyway
+        if (p.head_dim == 128) return launch_decode_d<128>(p, q, kv_pool, out, lse, stream);
+        if (p.head_dim == 64) return launch_decode_d<64>(p, q, kv_pool, out, lse, stream);
+        return cudaErrorInvalidValue;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace asynclm

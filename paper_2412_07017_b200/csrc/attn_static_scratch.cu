@@ -75,8 +75,7 @@ extern "C" int asynclm_attn_mixed_static(const asynclm_plan_t* plan, const void*
     d.partial_o = (float*)base;
     d.partial_lse = (float*)((unsigned char*)base + o_bytes);
     cudaStream_t s = (cudaStream_t)stream;
-    if (launch_attn_append_tc(d, q, kv_pool, out, lse, s) != cudaSuccess ||
-        launch_attn_decode(d, q, kv_pool, out, lse, s) != cudaSuccess ||
+    if (launch_attention(d, q, kv_pool, out, lse, s) != cudaSuccess ||
         launch_lse_merge(d, out, lse, s) != cudaSuccess) {
         (void)cudaGetLastError();
         return ASYNCLM_ERR_CUDA;

@@ -205,6 +205,107 @@ void cut_and_deal(const std::vector<int>& unit_ids, std::vector<UnitBuild>& unit
     cta_indptr[(size_t)n_ctas] = at;
 }
 
+
+// Measured costs of the attention kernels on B200, in nanoseconds, used only to balance CTAs.
+struct PathCost {
+    int gran;            // tokens per tile of the path (cuts fall on multiples of it)
+    int64_t tile_ns;     // one tile in steady state
+    int64_t item_ns;     // starting and finishing an item (pipeline fill and drain, merge, write)
+    int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
+};
+// (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
+constexpr PathCost kTensorCost{128, 1820, 5000, 3600};
+constexpr PathCost kCudaCost{96, 1250, 1200, 8500};
+
+// Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
+// then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
+// measured costs, and the line is cut into n_ctas nearly equal pieces.  A unit is split only where a
+// piece boundary falls inside it, so there are at most n_ctas - 1 more items than units, most CTAs
+// run one kind of work only, and the two kinds finish together.
+void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& ids_cuda,
+                  std::vector<UnitBuild>& units, int n_ctas, std::vector<Item>& items,
+                  std::vector<int32_t>& cta_indptr_cuda, std::vector<int32_t>& cta_indptr_tensor,
+                  std::vector<int32_t>& item_cta) {
+    struct Piece { Item it; int32_t cta; };
+    std::vector<Piece> best[2];
+    int64_t best_max = -1;
+    const std::vector<int>* ids[2] = {&ids_tensor, &ids_cuda};
+    const PathCost cost[2] = {kTensorCost, kCudaCost};
+    int64_t total = 0;
+    for (int path = 0; path < 2; ++path)
+        for (int id : *ids[path])
+            total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * cost[path].tile_ns;
+    total += (int64_t)n_ctas * (kTensorCost.item_ns + kCudaCost.phase_ns) / 2;
+    for (int round = 0; round < 4; ++round) {
+        const int64_t quota = std::max<int64_t>(1, (total + n_ctas - 1) / n_ctas);
+        std::vector<Piece> out[2];
+        std::vector<int64_t> load((size_t)n_ctas, 0);
+        int cta = 0;
+        int64_t cum = 0;      // cost laid down so far; CTA k ends where the line reaches (k + 1) * quota
+        bool has_phase[2] = {false, false};
+        auto next_cta = [&]() { ++cta; has_phase[0] = has_phase[1] = false; };
+        for (int path = 0; path < 2; ++path) {
+            const PathCost& pc = cost[path];
+            for (int id : *ids[path]) {
+                int64_t left = (units[id].n_keys + pc.gran - 1) / pc.gran;   // tiles left
+                int64_t k0 = 0;
+                int c = 0;
+                while (left > 0) {
+                    const bool last_cta = cta + 1 >= n_ctas;
+                    const int64_t start = pc.item_ns + (has_phase[path] ? 0 : pc.phase_ns);
+                    const int64_t room = (int64_t)(cta + 1) * quota - cum - start;
+                    int64_t take;
+                    if (last_cta || left * pc.tile_ns <= room + pc.item_ns) {
+                        take = left;                       // finishing here is cheaper than a new item elsewhere
+                    } else if (room < pc.tile_ns / 2 && load[(size_t)cta] > 0) {
+                        next_cta();
+                        continue;
+                    } else {
+                        take = std::max<int64_t>(1, (room + pc.tile_ns / 2) / pc.tile_ns);   // nearest: errors average out
+                    }
+                    const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
+                    out[path].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
+                    load[(size_t)cta] += start + take * pc.tile_ns;
+                    cum += start + take * pc.tile_ns;
+                    has_phase[path] = true;
+                    left -= take;
+                    k0 = k1;
+                    ++c;
+                    while (cta + 1 < n_ctas && cum >= (int64_t)(cta + 1) * quota) next_cta();
+                }
+            }
+        }
+        int64_t mx = 0, sum = 0;
+        for (int64_t l : load) { mx = std::max(mx, l); sum += l; }
+        if (best_max < 0 || mx < best_max) {
+            best_max = mx;
+            best[0] = out[0];
+            best[1] = out[1];
+        }
+        total = sum;      // the next round aims at the mean of what this round really cost
+    }
+    // emit: CUDA-core items first, then tensor items; chunk counts per unit
+    cta_indptr_cuda.assign((size_t)n_ctas + 1, 0);
+    cta_indptr_tensor.assign((size_t)n_ctas + 1, 0);
+    for (int path = 1; path >= 0; --path) {
+        std::vector<int32_t>& indptr = path == 1 ? cta_indptr_cuda : cta_indptr_tensor;
+        const int32_t first = (int32_t)items.size();
+        std::vector<int32_t> count((size_t)n_ctas, 0);
+        for (const Piece& pz : best[path]) {
+            items.push_back(pz.it);
+            item_cta.push_back(pz.cta);
+            count[(size_t)pz.cta]++;
+            units[pz.it.unit].u.n_chunks = pz.it.chunk + 1;
+        }
+        int32_t at = first;
+        for (int k = 0; k < n_ctas; ++k) {
+            indptr[(size_t)k] = at;
+            at += count[(size_t)k];
+        }
+        indptr[(size_t)n_ctas] = at;
+    }
+}
+
 }  // namespace
 
 extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_options* opts,
@@ -324,11 +425,17 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     const int ctas_tensor = n_sms;
     std::vector<Item> items;
     std::vector<int32_t> item_cta, cta_indptr_cuda, cta_indptr_tensor;
-    cut_and_deal(ids_cuda, units, fixed_chunk, ctas_cuda, kCudaItemOverheadTiles, items,
-                 cta_indptr_cuda, item_cta);
-    const int n_items_cuda = (int)items.size();
-    cut_and_deal(ids_tensor, units, fixed_chunk, ctas_tensor, kTensorItemOverheadTiles, items,
-                 cta_indptr_tensor, item_cta);
+    int n_items_cuda = 0;
+    if (fixed_chunk > 0 || ctas_cuda != ctas_tensor) {
+        cut_and_deal(ids_cuda, units, fixed_chunk, ctas_cuda, kCudaItemOverheadTiles, items,
+                     cta_indptr_cuda, item_cta);
+        n_items_cuda = (int)items.size();
+        cut_and_deal(ids_tensor, units, fixed_chunk, ctas_tensor, kTensorItemOverheadTiles, items,
+                     cta_indptr_tensor, item_cta);
+    } else {
+        deal_jointly(ids_tensor, ids_cuda, units, ctas_cuda, items, cta_indptr_cuda, cta_indptr_tensor, item_cta);
+        n_items_cuda = cta_indptr_cuda[(size_t)ctas_cuda];
+    }
     const int n_items = (int)items.size();
 
     // ---- partial rows ------------------------------------------------------------------------
@@ -444,8 +551,8 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     info.num_ctas_tensor = ctas_tensor;
     info.num_items_tensor = d.num_items_tensor;
     info.launches_append = T > 0 ? 1 : 0;
-    info.launches_attn = (n_items_cuda > 0 ? 1 : 0) + (d.num_items_tensor > 0 ? 1 : 0) +
-                         (d.num_split_units > 0 ? 1 : 0);
+    // span tiles and decode rows share one fused launch when a step has both (head_dim 128)
+    info.launches_attn = ((n_items_cuda > 0 || d.num_items_tensor > 0) ? 1 : 0) + (d.num_split_units > 0 ? 1 : 0);
     info.num_sms = n_sms;
     info.total_kv_tokens = total_kv;
     info.device_bytes_used = dev_need;
