@@ -30,6 +30,9 @@ if ROOT not in sys.path:
 METRIC = "kv_gbps_mixed_decode_interrupt_append"
 UNIT = "GB/s"
 WORKLOAD = "config2-llama3-8b-mixed-batch"
+# dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on this workload
+# (profiles/attn_fused_kernel_config2.md); None whenever the kernel has changed since that capture
+TRAFFIC_BYTES_PER_LAUNCH = 343_876_352
 
 
 def measured_peaks():
@@ -281,7 +284,7 @@ def run_gpu(args):
         tt = torch.tensor([e2e_total], device="cuda", dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         e2e_total = float(tt.item())
-    h2d = q_h.numel() * 2 + kn_h.numel() * 2 + vn_h.numel() * 2 + plan.info["device_bytes_used"] * 0
+    h2d = q_h.numel() * 2 + kn_h.numel() * 2 + vn_h.numel() * 2      # + the plan upload (tens of KB)
     d2h = out_h.numel() * 2
 
     if rank != 0:
@@ -312,12 +315,13 @@ def run_gpu(args):
             "plan": {k: plan.info[k] for k in ("num_items", "num_split_units", "num_items_tensor",
                                                "kv_chunk_tokens", "num_ctas_cuda", "num_ctas_tensor")},
         },
-        "roofline": {"bound": "hbm", "kernel": "asynclm_attn_mixed launches (attention + merge)",
+        "roofline": {"bound": "hbm",
+                     "kernel": "attn_fused_kernel (+ lse_merge_kernel; timed together as asynclm_attn_mixed)",
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None,
+                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH,
                      "algorithmic_bytes_per_launch": attn_bytes, "avg_launch_us": attn_s * 1e6},
         "e2e": {"value": world * by["kv"] / (e2e_total / e2e_steps) / 1e9, "unit": UNIT,
-                "h2d_bytes_per_step": int(h2d + plan.info["device_bytes_used"] * 0),
+                "h2d_bytes_per_step": int(h2d),
                 "d2h_bytes_per_step": int(d2h), "us_per_step": e2e_total / e2e_steps * 1e6,
                 "steps": e2e_steps, "includes": "H2D of q/k_new/v_new, asynclm_plan (+ its upload), "
                 "append, attention, D2H of out"},
