@@ -18,7 +18,11 @@
 //                   measured cost of about 90 cycles per small bulk/TMA copy made that the bottleneck.)
 //                   The two rings run independently so that a K tile never queues behind a V stage
 //                   that is still waiting for its P V to finish.
-//   warp 9          one thread issues the MMAs; the warp owns the tensor-memory allocation
+//   warps 9, 11     one thread each issues the Q K^T MMAs and the P V MMAs.  tcgen05.mma issue blocks
+//                   once a few MMAs are queued, so a single issuing thread alternates between being
+//                   blocked and doing its barrier bookkeeping while the tensor pipe idles; with two
+//                   issuers one's bookkeeping hides behind the other's MMAs.  Warp 9 owns the
+//                   tensor-memory allocation.
 // While one group runs the softmax of tile j the tensor core computes Q K^T of tile j+1 and P V of
 // tile j-1 for the other group.  All hand-offs are mbarriers with bounded waits; a wait that runs
 // out sets the plan's status word and a CTA-wide abort flag, every role falls through to the common
@@ -31,8 +35,8 @@ namespace asynclm {
 
 namespace tc {
 
-constexpr int kThreads = 352;
-constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10;
+constexpr int kThreads = 384;
+constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10, kMmaWarpPV = 11;
 constexpr int kD = 128;
 constexpr int kTile = 128;                       // keys per KV tile and query rows per tile
 constexpr int kKS = 2, kVS = 2;                  // ring depths
@@ -49,7 +53,7 @@ constexpr uint32_t kOffV = kOffK + kKS * kTileBytes;
 constexpr uint32_t kOffBar = kOffV + kVS * kTileBytes;
 enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPFull1, kPvDone0, kPvDone1, kSFull0, kSFull1, kKFull0,
            kKEmpty0 = kKFull0 + kKS, kVFull0 = kKEmpty0 + kKS, kVEmpty0 = kVFull0 + kVS,
-           kMmaDrain = kVEmpty0 + kVS, kNumBars };
+           kMmaDrain = kVEmpty0 + kVS, kMmaDrain2, kNumBars };
 constexpr uint32_t kOffTmemPtr = kOffBar + 8 * kNumBars;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
 constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
@@ -81,8 +85,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int32_t* status, int code) {
-    if (*abort_flag) return false;
     if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return false;
@@ -219,6 +223,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         for (int s = 0; s < kKS; ++s) { mbar_init(bar(kKFull0 + s), 32); mbar_init(bar(kKEmpty0 + s), 1); }
         for (int s = 0; s < kVS; ++s) { mbar_init(bar(kVFull0 + s), 32); mbar_init(bar(kVEmpty0 + s), 1); }
         mbar_init(bar(kMmaDrain), 1);
+        mbar_init(bar(kMmaDrain + 1), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
@@ -303,28 +308,31 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 while (!mbar_try_wait(bar(full0 + k % stages), (uint32_t)(k / stages) & 1u) && clock64() - t0 < kWaitCycles) {}
         }
     } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ Q K^T issuer
         if (lane == 0) {
             bool ok = true;
             int gt = 0;               // KV tiles issued so far (all items): ring position
-            int cnt[2] = {0, 0};      // tiles handed to each softmax group so far: S/P/PvDone phase
+            int cnt[2] = {0, 0};      // tiles handed to each softmax group so far: S/P phase
             int item_no = 0;
-            const uint32_t idesc_pv = instr_desc(128, 1);
             TItem it_next = load_titem(p, i0, i1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
                 it_next = load_titem(p, ii + 1, i1);      // in flight while this item runs
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
-                auto npages_of = [&](int j) {
-                    return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                };
-                // S[b] <- Q K_j^T for tile j of the item (b = j & 1); cnt[b] counts tiles of group b
-                auto issue_qk = [&](int j) {
+                ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
+                if (ok) tc_fence_after();
+                // S[b] <- Q K_j^T for tile j of the item (b = j & 1); S[b] is free once group b has turned
+                // its previous tile into P
+                for (int j = 0; j < ntiles && ok; ++j) {
                     const int g = gt + j, b = j & 1;
                     const int s = g % kKS;
-                    if (!mbar_wait(bar(kKFull0 + s), (uint32_t)(g / kKS) & 1u, abort_flag, p.status, 21)) return false;
+                    if (j >= 2)
+                        ok = mbar_wait(bar(kPFull0 + b), (uint32_t)(cnt[b] + (j >> 1) - 1) & 1u, abort_flag, p.status, 23);
+                    ok = ok && mbar_wait(bar(kKFull0 + s), (uint32_t)(g / kKS) & 1u, abort_flag, p.status, 21);
+                    if (!ok) break;
                     tc_fence_after();
-                    const uint32_t idesc = instr_desc(16u * (uint32_t)npages_of(j), 0);
+                    const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
+                    const uint32_t idesc = instr_desc(16u * (uint32_t)npg, 0);
                     const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
@@ -334,33 +342,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     }
                     mma_commit(bar(kKEmpty0 + s));
                     mma_commit(bar(kSFull0 + b));
-                    return true;
-                };
-                ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
-                if (!ok) break;
-                tc_fence_after();
-                ok = issue_qk(0);
-                if (ok && ntiles > 1) ok = issue_qk(1);
-                for (int j = 0; j < ntiles && ok; ++j) {
-                    const int g = gt + j, b = j & 1;
-                    const int s = g % kVS;
-                    ok = mbar_wait(bar(kPFull0 + b), (uint32_t)(cnt[b] + (j >> 1)) & 1u, abort_flag, p.status, 23) &&
-                         mbar_wait(bar(kVFull0 + s), (uint32_t)(g / kVS) & 1u, abort_flag, p.status, 24);
-                    if (ok && j == 0 && item_no > 0)
-                        ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const int npg = npages_of(j);
-                    for (int ks = 0; ks < npg; ++ks) {
-                        const uint32_t poff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        mma_f16(tmem + kColO + 128u * (uint32_t)b,
-                                smem_desc(sbase + kOffP + b * kTileBytes + poff, 16, 1024),
-                                smem_desc(sbase + kOffV + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
-                                idesc_pv, (j > 1 || ks > 0) ? 1u : 0u);
-                    }
-                    mma_commit(bar(kVEmpty0 + s));
-                    mma_commit(bar(kPvDone0 + b));
-                    if (j + 2 < ntiles) ok = issue_qk(j + 2);
                 }
                 gt += ntiles;
                 cnt[0] += (ntiles + 1) >> 1;
@@ -370,6 +351,50 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             mma_commit(bar(kMmaDrain));
             const long long t0 = clock64();
             while (!mbar_try_wait(bar(kMmaDrain), 0) && clock64() - t0 < kWaitCycles) {}
+        }
+        __syncwarp();
+      } else if (warp == kMmaWarpPV) {
+        // ------------------------------------------------------------------ P V issuer
+        if (lane == 0) {
+            bool ok = true;
+            int gt = 0;
+            int cnt[2] = {0, 0};
+            int item_no = 0;
+            const uint32_t idesc_pv = instr_desc(128, 1);
+            TItem it_next = load_titem(p, i0, i1);
+            for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
+                const TItem it = it_next;
+                it_next = load_titem(p, ii + 1, i1);
+                const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
+                // O[b] (+)= P_j V_j: P[b] comes from group b, V from the ring; the first P V into each
+                // accumulator of an item overwrites it, so the previous item's epilogue must be done
+                for (int j = 0; j < ntiles && ok; ++j) {
+                    const int g = gt + j, b = j & 1;
+                    const int s = g % kVS;
+                    ok = mbar_wait(bar(kPFull0 + b), (uint32_t)(cnt[b] + (j >> 1)) & 1u, abort_flag, p.status, 26) &&
+                         mbar_wait(bar(kVFull0 + s), (uint32_t)(g / kVS) & 1u, abort_flag, p.status, 24);
+                    if (ok && j == 0 && item_no > 0)
+                        ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
+                    for (int ks = 0; ks < npg; ++ks) {
+                        const uint32_t poff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                        mma_f16(tmem + kColO + 128u * (uint32_t)b,
+                                smem_desc(sbase + kOffP + b * kTileBytes + poff, 16, 1024),
+                                smem_desc(sbase + kOffV + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
+                                idesc_pv, (j > 1 || ks > 0) ? 1u : 0u);
+                    }
+                    mma_commit(bar(kVEmpty0 + s));
+                    mma_commit(bar(kPvDone0 + b));
+                }
+                gt += ntiles;
+                cnt[0] += (ntiles + 1) >> 1;
+                cnt[1] += ntiles >> 1;
+            }
+            mma_commit(bar(kMmaDrain + 1));
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar(kMmaDrain + 1), 0) && clock64() - t0 < kWaitCycles) {}
         }
         __syncwarp();
       }

@@ -214,8 +214,8 @@ struct PathCost {
     int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
 };
 // (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
-constexpr PathCost kTensorCost{128, 1820, 5000, 3600};
-constexpr PathCost kCudaCost{96, 1250, 1200, 8500};
+constexpr PathCost kTensorCost{128, 1590, 4500, 4800};
+constexpr PathCost kCudaCost{96, 1260, 1100, 6000};
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
 // then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
@@ -236,8 +236,8 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
         for (int id : *ids[path])
             total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * cost[path].tile_ns;
     total += (int64_t)n_ctas * (kTensorCost.item_ns + kCudaCost.phase_ns) / 2;
-    for (int round = 0; round < 4; ++round) {
-        const int64_t quota = std::max<int64_t>(1, (total + n_ctas - 1) / n_ctas);
+    int64_t quota = std::max<int64_t>(1, (total + n_ctas - 1) / n_ctas);
+    for (int round = 0; round < 8; ++round) {
         std::vector<Piece> out[2];
         std::vector<int64_t> load((size_t)n_ctas, 0);
         int cta = 0;
@@ -282,7 +282,12 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
             best[0] = out[0];
             best[1] = out[1];
         }
-        total = sum;      // the next round aims at the mean of what this round really cost
+        // next round: aim at the mean of what this round really cost; if the last CTA, which takes
+        // whatever is left, still ends up above the others, spread its excess over all of them
+        const int64_t mean = (sum + n_ctas - 1) / n_ctas;
+        const int64_t over = load[(size_t)n_ctas - 1] - quota;
+        quota = round == 0 ? mean : quota + (over > 0 ? (over + n_ctas - 1) / n_ctas : 0);
+        if (round > 0 && over <= 0) break;
     }
     // emit: CUDA-core items first, then tensor items; chunk counts per unit
     cta_indptr_cuda.assign((size_t)n_ctas + 1, 0);
