@@ -106,14 +106,26 @@ def bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
     return u.view(np.float32).astype(np.float64)
 
 
-def normal_bf16(seed: int, stream: int, shape: Sequence[int], chunk: int = 1 << 24) -> np.ndarray:
-    """N(0,1) samples rounded to bf16, drawn in fixed-size chunks from one Philox stream."""
+def normal_bf16(seed: int, stream: int, shape: Sequence[int], chunk: int = 1 << 22) -> np.ndarray:
+    """N(0,1) samples rounded to bf16.  Chunk c of a tensor comes from its own Philox stream keyed by
+    (seed, stream, c), so chunks can be drawn in parallel and any slice can be redrawn."""
     n = int(np.prod(shape))
     out = np.empty(n, dtype=np.uint16)
-    g = _rng(seed, stream)
-    for s in range(0, n, chunk):
-        e = min(n, s + chunk)
+
+    def fill(c: int) -> None:
+        s, e = c * chunk, min(n, (c + 1) * chunk)
+        g = np.random.Generator(np.random.Philox(key=[int(seed) & (2**64 - 1), (int(stream) << 24) | c]))
         out[s:e] = f32_to_bf16_bits(g.standard_normal(e - s, dtype=np.float32))
+
+    nchunks = (n + chunk - 1) // chunk
+    if nchunks <= 2:
+        for c in range(nchunks):
+            fill(c)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        import os
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
+            list(ex.map(fill, range(nchunks)))
     return out.reshape(tuple(shape))
 
 
