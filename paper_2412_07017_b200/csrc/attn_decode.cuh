@@ -29,7 +29,10 @@ namespace dec {
 constexpr int kWarps = 12;                   // consumer warps (three warpgroups)
 constexpr int kThreads = (kWarps + 4) * 32;  // + the producer's warpgroup (one working warp)
 constexpr int kRowsPerWarp = 8;
-constexpr int kTileTok = kWarps * kRowsPerWarp;   // 96 rows per ring stage (6 pages)
+// A warp works on at most 4 query heads (the accumulators of more do not fit its registers).  With
+// 8 heads per kv head the warps split into two halves that take 4 heads each and share the K/V
+// rows in shared memory: 6 row blocks x 2 head halves, 48-row tiles instead of 96.
+__host__ __device__ constexpr int head_splits(int group) { return group > 4 ? group / 4 : 1; }
 // Register budget: the CTA is launched with 512 x 128 registers; the producer's warpgroup gives
 // most of its share back and the consumers take it: 384 x 160 + 128 x 24 = 64512 <= 65536.
 constexpr int kRegsConsumer = 160, kRegsProducer = 24;
@@ -120,7 +123,7 @@ __device__ __forceinline__ void transpose_reduce(float (&v)[NMAX]) {
 
 constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
 
-template <int D, int G>
+template <int D, int G, int HS = 1>     // G: heads per warp, HS: head halves per CTA
 struct Geometry {
     static constexpr int LPR = D / 8;                 // lanes per row (16 bytes each)
     static constexpr int TPW = 32 / LPR;              // rows per warp-wide shared-memory load
@@ -129,9 +132,11 @@ struct Geometry {
     static constexpr int NF = NV >= LPR ? NV / LPR : 1;              // finished scores per lane
     static constexpr int DUP_SHIFT = NV >= LPR ? 0 : ilog2(LPR / NV); // lanes holding duplicates
     static constexpr int PAGE_BYTES = kPage * D * 2;
-    static constexpr int TILE_BYTES = (kTileTok / kPage) * PAGE_BYTES;   // K (or V) part of a stage
+    static constexpr int ROW_BLOCKS = kWarps / HS;
+    static constexpr int TILE_TOK = ROW_BLOCKS * kRowsPerWarp;          // rows per ring stage: 96 or 48
+    static constexpr int TILE_BYTES = (TILE_TOK / kPage) * PAGE_BYTES;   // K (or V) part of a stage
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
-    static constexpr int Q_BYTES = G * D * 2;
+    static constexpr int Q_BYTES = G * HS * D * 2;
     static constexpr int STAT_FLOATS = (kWarps * G + 7) / 8 * 8;         // max (or sum) array, padded to 32 bytes
     static constexpr int MERGE_FLOATS = 2 * STAT_FLOATS + kWarps * G * D;  // one merge buffer
     // A lane's slot (i, g) holds the partial score of true row i ^ xi and true head g ^ xg, with
@@ -144,22 +149,25 @@ struct Geometry {
     __host__ __device__ static constexpr int score_slot(int i, int g) { return NV >= LPR ? (i * G + g) % NF : 0; }
 };
 
-template <int D, int G>
+template <int D, int GT>
 size_t smem_bytes(int stages) {
-    using Geo = Geometry<D, G>;
+    using Geo = Geometry<D, GT / head_splits(GT), head_splits(GT)>;
     return (size_t)stages * (Geo::STAGE_BYTES + Geo::Q_BYTES + sizeof(TileDesc) + 16) +
            2 * Geo::MERGE_FLOATS * sizeof(float) + 3 * 8 + 16 + 1024;
 }
 
 // The whole kernel body.  FUSED: the CTA has just finished the tensor-core phase of the fused
 // kernel, in which warps 0-7 held 168 registers, warps 8-11 held 80 and warps 12-15 held 24.
-template <int D, int G, bool FUSED>
+template <int D, int GT, bool FUSED>
 __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
                                             const __nv_bfloat16* __restrict__ pool,
                                             __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                                             int S, uint8_t* smem) {
-    using Geo = Geometry<D, G>;
+    constexpr int HS = head_splits(GT);     // head halves
+    constexpr int G = GT / HS;              // query heads per warp
+    using Geo = Geometry<D, G, HS>;
     constexpr int LPR = Geo::LPR, TPW = Geo::TPW, NR = Geo::NR, NV = Geo::NV, NF = Geo::NF;
+    constexpr int RB = Geo::ROW_BLOCKS, kTileTok = Geo::TILE_TOK;
     uint8_t* stage_base = smem;
     uint8_t* q_base = stage_base + (size_t)S * Geo::STAGE_BYTES;
     float* merge_base = (float*)(q_base + (size_t)S * Geo::Q_BYTES);
@@ -257,7 +265,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
                         bulk_g2s(dst + Geo::TILE_BYTES, src + (size_t)Hkv * kPage * D, Geo::PAGE_BYTES, full0 + 8 * s);
                     }
                     if (first && lane == 31) {
-                        const __nv_bfloat16* src = q + ((size_t)cur.q_row0 * Hq + (size_t)cur.kv_head * G) * D;
+                        const __nv_bfloat16* src = q + ((size_t)cur.q_row0 * Hq + (size_t)cur.kv_head * GT) * D;
                         bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
                     }
                 }
@@ -317,7 +325,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
             const uint8_t* qs = q_base + (size_t)s * Geo::Q_BYTES;
 #pragma unroll
             for (int g = 0; g < G; ++g) {
-                const uint4 w = *reinterpret_cast<const uint4*>(qs + ((size_t)(g ^ xg) * D + sub * 8) * 2);
+                const uint4 w = *reinterpret_cast<const uint4*>(qs + ((size_t)((warp / RB) * G + (g ^ xg)) * D + sub * 8) * 2);
                 q2[g][0] = unpack2(w.x); q2[g][1] = unpack2(w.y);
                 q2[g][2] = unpack2(w.z); q2[g][3] = unpack2(w.w);
 #pragma unroll
@@ -332,7 +340,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
             cur_out_row = d.out_row; cur_kv_head = d.kv_head; cur_partial = d.partial_row;
         }
         const int rows = d.rows;
-        const int blk = warp;
+        const int blk = warp % RB;      // row block of the tile; warp / RB is the head half
         const bool active = blk * kRowsPerWarp < rows;
         uint4 kw[NR], vw[NR];
         if (active) {
@@ -474,14 +482,16 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
             if (!mbar_wait(mb, (uint32_t)(item_count >> 1) & 1u, abort_flag, p.status, 3)) break;
             ++item_count;
             const int tid = threadIdx.x;
-            for (int e = 2 * tid; e < G * D; e += 2 * kWarps * 32) {
-                const int g = e / D, dd = e % D;
+            for (int e = 2 * tid; e < GT * D; e += 2 * kWarps * 32) {
+                const int gfull = e / D, dd = e % D;
+                const int g = gfull % G, w0 = (gfull / G) * RB;      // the RB warps that hold this head
                 float M = -INFINITY;
 #pragma unroll
-                for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mm[w * G + g]);
+                for (int r = 0; r < RB; ++r) M = fmaxf(M, mm[(w0 + r) * G + g]);
                 float L = 0.f, a0 = 0.f, a1 = 0.f;
 #pragma unroll
-                for (int w = 0; w < kWarps; ++w) {
+                for (int r = 0; r < RB; ++r) {
+                    const int w = w0 + r;
                     const float wgt = fast_exp2(mm[w * G + g] - M);
                     L = fmaf(ml[w * G + g], wgt, L);
                     const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * G + g) * D + dd);
@@ -489,16 +499,16 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
                     a1 = fmaf(ov.y, wgt, a1);
                 }
                 const float inv = 1.f / L;
-                const size_t hq = (size_t)cur_kv_head * G + g;
+                const size_t hq = (size_t)cur_kv_head * GT + gfull;
                 if (cur_partial < 0) {
                     *reinterpret_cast<uint32_t*>(out + ((size_t)cur_out_row * Hq + hq) * D + dd) =
                         pack_bf16x2(a0 * inv, a1 * inv);
                     if (lse != nullptr && dd == 0)
                         lse[(size_t)cur_out_row * Hq + hq] = (M + log2f(L)) * kLn2;
                 } else {
-                    *reinterpret_cast<float2*>(p.partial_o + ((size_t)cur_partial * G + g) * D + dd) =
+                    *reinterpret_cast<float2*>(p.partial_o + ((size_t)cur_partial * GT + gfull) * D + dd) =
                         make_float2(a0 * inv, a1 * inv);
-                    if (dd == 0) p.partial_lse[(size_t)cur_partial * G + g] = M + log2f(L);
+                    if (dd == 0) p.partial_lse[(size_t)cur_partial * GT + gfull] = M + log2f(L);
                 }
             }
         }
