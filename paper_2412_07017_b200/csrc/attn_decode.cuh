@@ -19,6 +19,8 @@
 // Every wait is bounded: a wait that runs out sets the plan's device status word and a CTA-wide
 // abort flag, after which all loops fall through and the kernel returns.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -96,6 +98,17 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
+// One tiled TMA copy fetches the K block and the V block of a (page, kv head): the pool is described
+// to the TMA unit as a 5-D tensor [pages][2][Hkv][16][d] and the box spans (d, 16, 1, 2, 1), i.e. two
+// separate 16 x d blocks of global memory that land back to back in shared memory.  (A bulk/TMA
+// copy costs about 70 cycles plus 1 cycle per 107 bytes on this part, so halving the number of
+// copies matters.)  No multicast.
+__device__ __forceinline__ void tma_page_kv(uint32_t dst, const CUtensorMap* map, int kv_head, int page, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(0), "r"(0), "r"(kv_head), "r"(0), "r"(page), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
 
 // Transposing reduction over the LPR lanes that share a row.  Every lane starts with N values that
@@ -134,8 +147,8 @@ struct Geometry {
     static constexpr int PAGE_BYTES = kPage * D * 2;
     static constexpr int ROW_BLOCKS = kWarps / HS;
     static constexpr int TILE_TOK = ROW_BLOCKS * kRowsPerWarp;          // rows per ring stage: 96 or 48
-    static constexpr int TILE_BYTES = (TILE_TOK / kPage) * PAGE_BYTES;   // K (or V) part of a stage
-    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    // a stage holds, page after page, the page's K block followed by its V block
+    static constexpr int STAGE_BYTES = (TILE_TOK / kPage) * 2 * PAGE_BYTES;
     static constexpr int Q_BYTES = G * HS * D * 2;
     static constexpr int STAT_FLOATS = (kWarps * G + 7) / 8 * 8;         // max (or sum) array, padded to 32 bytes
     static constexpr int MERGE_FLOATS = 2 * STAT_FLOATS + kWarps * G * D;  // one merge buffer
@@ -159,8 +172,8 @@ size_t smem_bytes(int stages) {
 // The whole kernel body.  FUSED: the CTA has just finished the tensor-core phase of the fused
 // kernel, in which warps 0-7 held 168 registers, warps 8-11 held 80 and warps 12-15 held 24.
 template <int D, int GT, bool FUSED>
-__device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
-                                            const __nv_bfloat16* __restrict__ pool,
+__device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap* kv_map,
+                                            const __nv_bfloat16* __restrict__ q,
                                             __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                                             int S, uint8_t* smem) {
     constexpr int HS = head_splits(GT);     // head halves
@@ -192,7 +205,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
     }
     __syncthreads();
 
-    const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+    const int Hq = p.num_q_heads;
 
     if (warp >= kWarps) {
         if constexpr (!FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
@@ -258,12 +271,9 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
                     __syncwarp();
                     const int64_t page = __shfl_sync(0xffffffffu, pages_cur,
                                                      (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
-                    if (lane < npages) {
-                        const __nv_bfloat16* src = pool + pool_row_offset(page, 0, cur.kv_head, 0, Hkv, D);
-                        const uint32_t dst = smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * Geo::PAGE_BYTES);
-                        bulk_g2s(dst, src, Geo::PAGE_BYTES, full0 + 8 * s);
-                        bulk_g2s(dst + Geo::TILE_BYTES, src + (size_t)Hkv * kPage * D, Geo::PAGE_BYTES, full0 + 8 * s);
-                    }
+                    if (lane < npages)
+                        tma_page_kv(smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * 2 * Geo::PAGE_BYTES),
+                                    kv_map, cur.kv_head, (int)page, full0 + 8 * s);
                     if (first && lane == 31) {
                         const __nv_bfloat16* src = q + ((size_t)cur.q_row0 * Hq + (size_t)cur.kv_head * GT) * D;
                         bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
@@ -344,12 +354,13 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const __nv_bfloat1
         const bool active = blk * kRowsPerWarp < rows;
         uint4 kw[NR], vw[NR];
         if (active) {
-            const uint8_t* ks = stage_base + (size_t)s * Geo::STAGE_BYTES +
-                                (size_t)(blk * kRowsPerWarp) * (D * 2) + lane * 16;
+            // the warp's 8 rows are one half of a page: [page][K 16 rows | V 16 rows]
+            const uint8_t* ks = stage_base + (size_t)s * Geo::STAGE_BYTES + (size_t)(blk >> 1) * 2 * Geo::PAGE_BYTES +
+                                (size_t)((blk & 1) * kRowsPerWarp) * (D * 2) + lane * 16;
 #pragma unroll
             for (int i = 0; i < NR; ++i) {
                 kw[i] = *reinterpret_cast<const uint4*>(ks + (size_t)(i ^ xi) * TPW * D * 2);
-                vw[i] = *reinterpret_cast<const uint4*>(ks + Geo::TILE_BYTES + (size_t)(i ^ xi) * TPW * D * 2);
+                vw[i] = *reinterpret_cast<const uint4*>(ks + Geo::PAGE_BYTES + (size_t)(i ^ xi) * TPW * D * 2);
             }
         }
         __syncwarp();

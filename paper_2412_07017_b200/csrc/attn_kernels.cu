@@ -25,11 +25,11 @@ __device__ __forceinline__ uint8_t* aligned_smem(uint8_t* raw) {
 
 template <int D, int G>
 __global__ void __launch_bounds__(dec::kThreads, 1)
-attn_decode_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pool,
+attn_decode_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const __nv_bfloat16* __restrict__ q,
                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
     extern __shared__ uint8_t smem_raw[];
     pdl_wait();
-    dec::decode_body<D, G, false>(p, q, pool, out, lse, S, aligned_smem(smem_raw));
+    dec::decode_body<D, G, false>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw));
 }
 
 template <int G>
@@ -42,13 +42,42 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv
 
 template <int G>
 __global__ void __launch_bounds__(dec::kThreads, 1)
-attn_fused_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pool,
-                  __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
+attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const __nv_bfloat16* __restrict__ q,
+                  const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+                  int S) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = aligned_smem(smem_raw);
     tc::tc_body<G, true>(p, q, pool, out, lse, smem);
     __syncthreads();      // tensor memory released, shared memory free for the second phase
-    dec::decode_body<tc::kD, G, true>(p, q, pool, out, lse, S, smem);
+    dec::decode_body<tc::kD, G, true>(p, &kv_map, q, out, lse, S, smem);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The pool as a 5-D tensor (d, 16 slots, Hkv, K|V, pages) with a box of one page's K and V blocks of
+// one kv head (see dec::tma_page_kv).  The driver entry point is looked up once per process.
+cudaError_t make_kv_map(const DevPlan& p, const void* pool, CUtensorMap* map) {
+    static EncodeTiledFn encode = nullptr;
+    if (encode == nullptr) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+        encode = (EncodeTiledFn)sym;
+    }
+    const cuuint64_t d = (cuuint64_t)p.head_dim, hkv = (cuuint64_t)p.num_kv_heads;
+    if (p.num_pages <= 0 || p.num_pages > 0x7fffffff) return cudaErrorInvalidValue;
+    const cuuint64_t dims[5] = {d, kPage, hkv, 2, (cuuint64_t)p.num_pages};
+    const cuuint64_t strides[4] = {d * 2, kPage * d * 2, hkv * kPage * d * 2, 2 * hkv * kPage * d * 2};
+    const cuuint32_t box[5] = {(cuuint32_t)d, kPage, 1, 2, 1};
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box,
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
 template <int D, int G>
@@ -65,8 +94,11 @@ cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, voi
     const size_t smem = dec::smem_bytes<D, G>(S);
     cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_decode_kernel<D, G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p,
-                      (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
+    CUtensorMap map;
+    e = make_kv_map(p, pool, &map);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(attn_decode_kernel<D, G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p, map,
+                      (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, S);
 }
 
 template <int G>
@@ -86,7 +118,10 @@ cudaError_t launch_fused(const DevPlan& p, const void* q, const void* pool, void
     const size_t smem = dec::smem_bytes<tc::kD, G>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD, G>(S) : tc::kSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_fused_kernel<G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p,
+    CUtensorMap map;
+    e = make_kv_map(p, pool, &map);
+    if (e != cudaSuccess) return e;
+    return launch_pdl(attn_fused_kernel<G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p, map,
                       (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
 }
 
