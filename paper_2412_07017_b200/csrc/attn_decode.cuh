@@ -37,7 +37,7 @@ constexpr int kRowsPerWarp = 8;
 __host__ __device__ constexpr int head_splits(int group) { return group > 4 ? group / 4 : 1; }
 // Register budget: the CTA is launched with 512 x 128 registers; the producer's warpgroup gives
 // most of its share back and the consumers take it: 384 x 160 + 128 x 24 = 64512 <= 65536.
-constexpr int kRegsConsumer = 160, kRegsProducer = 24;
+constexpr int kRegsConsumer = 152, kRegsProducer = 56;
 static_assert(kWarps * 32 * kRegsConsumer + 128 * kRegsProducer <= 65536, "register split");
 constexpr float kRescaleThreshold = 16.f;    // log2 units a score may exceed the reference max by
 constexpr long long kWaitCycles = 2000000000ll;
