@@ -1,32 +1,37 @@
-// Tensor-core attention for interrupt spans (tcgen05 MMA with accumulators in tensor memory).
+// Tensor-core attention for interrupt spans (tcgen05 MMA, accumulators and P in tensor memory).
 //
 // An interrupt span is a block of new tokens appended to one sequence (paper Section 3.2); in the
 // next decoding step (Section 5.3) every token of the span attends to the whole cached context and
 // causally to the span itself.  With G query heads per kv head, a span of q tokens gives G*q query
 // rows against the same K/V, which is a dense contraction: rows are packed 128 to a tile
-// (row m = token m / G, head m % G) and S = Q K^T and O += P V run on the tensor cores.
+// (row r = token r / G, head r % G) and S = Q K^T and O += P V run on the tensor cores.
 //
-// One persistent CTA per SM, ten warps:
-//   warps 0-3, 4-7  two softmax groups, one thread per query row each.  Group b takes the KV tiles
-//                   j = b, b+2, ... of an item and owns S[b], P[b] and O[b]: softmax on S read from
-//                   tensor memory, P written to shared memory as bf16, lazy rescaling of O[b].  The
-//                   two running (max, sum, O) states are merged in the epilogue like two KV splits.
-//   warps 8, 10     producers of the K ring and of the V ring: 16-byte cp.async copies (fully coalesced,
+// A work item covers up to 256 query rows (two row tiles) of one (sequence, kv head) and a range of
+// keys.  One persistent CTA per SM, twelve working warps:
+//   warps 0-3, 4-7  two softmax groups, one thread per query row of a tile.  Each group owns one S
+//                   accumulator (128 fp32 columns of tensor memory) and one O accumulator.
+//                     * items with more than 128 rows ("dual"): group b owns row tile b and both
+//                       groups consume every KV tile, so K and V are fetched once for 256 rows;
+//                     * items with at most 128 rows: the groups take alternate KV tiles of the one
+//                       row tile and their (max, sum, O) states are merged in the epilogue like two
+//                       KV splits.
+//                   The softmax runs in place: a thread reads its row of S 32 columns at a time and
+//                   writes P as packed bf16 pairs over the columns it has already read; P V then
+//                   takes its A operand from tensor memory.  The reference maximum only moves when
+//                   a score exceeds it by 2^8; then O, the running sum and the part of P already
+//                   written are rescaled.
+//   warps 8, 10     producers of K tiles and of V tiles: 16-byte cp.async copies (fully coalesced,
 //                   two 256-byte rows per warp instruction) that write the 128-byte-swizzled operand
-//                   layout directly and complete on the stage's mbarrier; rows behind the last key are
-//                   zero-filled.  (Tiled TMA would need 32 boxes of 2 KiB per 128-key tile, and the
-//                   measured cost of about 90 cycles per small bulk/TMA copy made that the bottleneck.)
-//                   The two rings run independently so that a K tile never queues behind a V stage
-//                   that is still waiting for its P V to finish.
-//   warps 9, 11     one thread each issues the Q K^T MMAs and the P V MMAs.  tcgen05.mma issue blocks
-//                   once a few MMAs are queued, so a single issuing thread alternates between being
-//                   blocked and doing its barrier bookkeeping while the tensor pipe idles; with two
-//                   issuers one's bookkeeping hides behind the other's MMAs.  Warp 9 owns the
+//                   layout and complete on the slot's mbarrier.  K and V share one ring of five
+//                   32 KiB slots, filled in the order the tensor core consumes them
+//                   (K0 K1 V0 K2 V1 K3 ...): a V tile is needed one softmax later than the K tile
+//                   of the same keys, and a shared ring lets whichever is due use the free slots.
+//   warps 9, 11     one thread each issues the Q K^T MMAs and the P V MMAs (two issuers, so that
+//                   one's barrier bookkeeping hides behind the other's MMAs).  Warp 9 owns the
 //                   tensor-memory allocation.
-// While one group runs the softmax of tile j the tensor core computes Q K^T of tile j+1 and P V of
-// tile j-1 for the other group.  All hand-offs are mbarriers with bounded waits; a wait that runs
-// out sets the plan's status word and a CTA-wide abort flag, every role falls through to the common
-// exit, and the tensor memory is released there.
+// All hand-offs are mbarriers with bounded waits; a wait that runs out sets the plan's status word
+// and a CTA-wide abort flag, every role falls through to the common exit, and the tensor memory is
+// released there.
 #pragma once
 #include "common.cuh"
 #include "kernels.h"
@@ -38,31 +43,36 @@ namespace tc {
 constexpr int kThreads = 384;
 constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10, kMmaWarpPV = 11;
 constexpr int kD = 128;
-constexpr int kTile = 128;                       // keys per KV tile and query rows per tile
-constexpr int kKS = 2, kVS = 2;                  // ring depths
+constexpr int kTile = 128;                       // keys per K/V ring slot and query rows per row tile
+constexpr int kSub = 64;                         // keys per softmax step (one S buffer)
+constexpr int kRing = 5;                         // K/V ring slots
 constexpr uint32_t kHalfBytes = 128 * 128;       // one 64-value half of a 128-row tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;  // 32 KiB
 constexpr float kRescaleThreshold = 8.f;
 constexpr long long kWaitCycles = 2000000000ll;
 
 // shared memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffP = kOffQ + kTileBytes;          // P[0], P[1]
-constexpr uint32_t kOffK = kOffP + 2 * kTileBytes;
-constexpr uint32_t kOffV = kOffK + kKS * kTileBytes;
-constexpr uint32_t kOffBar = kOffV + kVS * kTileBytes;
-enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPFull1, kPvDone0, kPvDone1, kSFull0, kSFull1, kKFull0,
-           kKEmpty0 = kKFull0 + kKS, kVFull0 = kKEmpty0 + kKS, kVEmpty0 = kVFull0 + kVS,
-           kMmaDrain = kVEmpty0 + kVS, kMmaDrain2, kNumBars };
+constexpr uint32_t kOffQ = 0;                           // Q[0], Q[1]
+constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
+constexpr uint32_t kOffBar = kOffRing + kRing * kTileBytes;
+// S, P V and P hand-offs exist per (group b, S buffer): index 2 * b + buffer
+enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPvDone0 = kPFull0 + 4, kSFull0 = kPvDone0 + 4,
+           kRingFull0 = kSFull0 + 4, kRingEmpty0 = kRingFull0 + kRing, kMmaDrain = kRingEmpty0 + kRing,
+           kMmaDrain2, kNumBars };
 constexpr uint32_t kOffTmemPtr = kOffBar + 8 * kNumBars;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
 constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
 // tensor memory columns
-constexpr uint32_t kColS = 0;      // S[0], S[1]: 128 columns each
+constexpr uint32_t kColS = 0;      // group b: two S buffers of 64 columns each at 128 b + 64 buffer; the P of a
+                                   // buffer overlays its first 32 columns
 constexpr uint32_t kColO = 256;    // O[0], O[1]: 128 columns each
 constexpr uint32_t kTmemCols = 512;
+
+// Ring position of the K tile and of the V tile of the CTA's g-th KV tile: K0 K1 V0 K2 V1 K3 ...
+__device__ __forceinline__ int ring_pos_k(int g) { return g == 0 ? 0 : 2 * g - 1; }
+__device__ __forceinline__ int ring_pos_v(int g) { return 2 * g + 2; }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -166,25 +176,56 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// 16 consecutive 32-bit columns of this warp's 32 rows.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld2(uint32_t taddr, uint32_t& a, uint32_t& b) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(a), "=r"(b) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st2(uint32_t taddr, uint32_t a, uint32_t b) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%2], {%0,%1};" ::"r"(a), "r"(b), "r"(taddr) : "memory");
+}
+// D (+)= A B with A taken from tensor memory: row i of A is lane i, its 16 bf16 values of one K step
+// are 8 consecutive 32-bit columns (two values per column, the lower index in the low half).
+__device__ __forceinline__ void mma_f16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// One work item as the kernel sees it (kv_end == 0: no item).
 struct TItem {
-    int kv0, kv_end;      // key range of the item after causal clipping (kv_end == 0: no item)
-    int q_row0, ntok, kv_limit0, kv_head, partial_base, chunk, page0;
+    int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row0, page0;
 };
 
 __device__ __forceinline__ TItem load_titem(const DevPlan& p, int ii, int i1) {
-    TItem r{0, 0, 0, 0, 0, 0, -1, 0, 0};
+    TItem r{0, 0, 0, 0, 0, 0, -1, 0};
     if (ii < i1) {
-        const Item it = p.items[ii];
-        const Unit u = p.units[it.unit];
-        r.kv0 = it.kv0;
-        r.kv_end = min(it.kv1, u.kv_limit0 + u.ntok - 1);
-        r.q_row0 = u.q_row0;
-        r.ntok = u.ntok;
-        r.kv_limit0 = u.kv_limit0;
-        r.kv_head = u.kv_head;
-        r.partial_base = u.partial_base;
-        r.chunk = it.chunk;
-        r.page0 = u.page_base + it.kv0 / kPage;
+        const int4* src = reinterpret_cast<const int4*>(p.works + ii);
+        const int4 a = __ldg(src), b = __ldg(src + 1);
+        r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z; r.ntok = a.w;
+        r.kv_limit0 = b.x; r.kv_head = b.y; r.partial_row0 = b.z; r.page0 = b.w;
     }
     return r;
 }
@@ -194,7 +235,7 @@ __device__ __forceinline__ TItem load_titem(const DevPlan& p, int ii, int i1) {
 constexpr int kRegsSoftmaxFused = 168, kRegsIssueFused = 80, kRegsIdleFused = 24;
 static_assert(256 * kRegsSoftmaxFused + 128 * kRegsIssueFused + 128 * kRegsIdleFused <= 65536, "register split");
 
-// The whole kernel body.  FUSED: called by all 16 warps of the fused kernel (warps 11-15 only take
+// The whole kernel body.  FUSED: called by all 16 warps of the fused kernel (warps 12-15 only take
 // part in the CTA-wide barriers), with `smem` 1024-byte aligned.
 template <int G, bool FUSED>
 __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
@@ -210,19 +251,20 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+    // The plan was uploaded before the kernel in front of this one started, so it may be read before
+    // pdl_wait(); everything else (pool, q, outputs) is touched only after it.
     const int i0 = p.cta_indptr_tensor[blockIdx.x], i1 = p.cta_indptr_tensor[blockIdx.x + 1];
 
     if (threadIdx.x == 0) {
         mbar_init(bar(kQFull), 256);
         mbar_init(bar(kStats), 256);
         mbar_init(bar(kOFree), 256);
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < 4; ++b) {
             mbar_init(bar(kPFull0 + b), 128);
             mbar_init(bar(kPvDone0 + b), 1);
             mbar_init(bar(kSFull0 + b), 1);
         }
-        for (int s = 0; s < kKS; ++s) { mbar_init(bar(kKFull0 + s), 32); mbar_init(bar(kKEmpty0 + s), 1); }
-        for (int s = 0; s < kVS; ++s) { mbar_init(bar(kVFull0 + s), 32); mbar_init(bar(kVEmpty0 + s), 1); }
+        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kRingFull0 + s), 32); mbar_init(bar(kRingEmpty0 + s), 1); }
         mbar_init(bar(kMmaDrain), 1);
         mbar_init(bar(kMmaDrain + 1), 1);
         *abort_flag = 0;
@@ -238,11 +280,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_ptr;
-    // Launched with programmatic serialization: everything above overlapped the tail of the append
-    // kernel; from here on the pool is read.  Once every CTA has passed this point the CUDA-core
-    // kernel behind this one may start on SMs that become free.
-    pdl_wait();
-    if constexpr (!FUSED) pdl_trigger();
 
     if (warp >= 12) {
         if constexpr (FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIdleFused));
@@ -250,10 +287,8 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
       if constexpr (FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssueFused));
       if (warp == kProducerWarpK || warp == kProducerWarpV) {
         // ------------------------------------------------------------------ producer warps
-        const int which = warp == kProducerWarpV ? 1 : 0;       // 0: K ring, 1: V ring
-        const int stages = which ? kVS : kKS;
-        const int full0 = which ? kVFull0 : kKFull0, empty0 = which ? kVEmpty0 : kKEmpty0;
-        const uint32_t ring = sbase + (which ? kOffV : kOffK);
+        const int which = warp == kProducerWarpV ? 1 : 0;       // 0: K tiles, 1: V tiles
+        const uint32_t ring = sbase + kOffRing;
         auto load_pages = [&](const TItem& it, int first_page) {
             const int npg = (it.kv_end - it.kv0 + kPage - 1) / kPage;
             const int idx = first_page + lane;
@@ -262,9 +297,11 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         constexpr int kPagesPerTile = kTile / kPage;          // 8
         constexpr int kGroupTiles = 32 / kPagesPerTile;       // 4
         bool ok = true;
-        int n = 0;                                             // tiles issued so far
+        int n = 0;                                             // KV tiles issued so far (all items)
+        int last_pos = -1;
         TItem cur = load_titem(p, i0, i1), nxt = load_titem(p, i0 + 1, i1);
         int pages_cur = cur.kv_end > 0 ? load_pages(cur, 0) : 0;
+        pdl_wait();
         for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
             const TItem after = load_titem(p, ii + 2, i1);
             const int ntiles = (cur.kv_end - cur.kv0 + kTile - 1) / kTile;
@@ -276,9 +313,11 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 for (int t = t0; t < t1 && ok; ++t, ++n) {
                     const int rows = min(kTile, cur.kv_end - (cur.kv0 + t * kTile));
                     const int npages = (rows + kPage - 1) / kPage;
-                    const int s = n % stages;
-                    ok = mbar_wait_warp(bar(empty0 + s), ((uint32_t)(n / stages) & 1u) ^ 1u, abort_flag, p.status, 11 + which);
+                    const int pos = which ? ring_pos_v(n) : ring_pos_k(n);
+                    const int s = pos % kRing;
+                    ok = mbar_wait_warp(bar(kRingEmpty0 + s), ((uint32_t)(pos / kRing) & 1u) ^ 1u, abort_flag, p.status, 11 + which);
                     if (!ok) break;
+                    last_pos = pos;
                     // lane -> 16-byte chunk c of row 2*rr + (lane >> 4) of each page: a warp instruction
                     // moves two whole 256-byte rows
                     const int c = lane & 15;
@@ -295,58 +334,66 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                                        src_page + slot * (kD * 2) + c * 16, row < rows ? 16u : 0u);
                         }
                     }
-                    cp_async_arrive(bar(full0 + s));
+                    cp_async_arrive(bar(kRingFull0 + s));
                 }
                 pages_cur = pages_nxt;
             }
             cur = nxt;
             nxt = after;
         }
-        if (!ok) {
+        if (!ok && last_pos >= 0) {
             // aborted: let the loads already issued land before shared memory goes away
-            const long long t0 = clock64();
-            for (int k = max(0, n - stages); k < n; ++k)
-                while (!mbar_try_wait(bar(full0 + k % stages), (uint32_t)(k / stages) & 1u) && clock64() - t0 < kWaitCycles) {}
+            asm volatile("cp.async.wait_all;" ::: "memory");
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ Q K^T issuer
+        // A KV tile is consumed in steps of 64 keys.  Step u of group b (counted over the CTA's whole
+        // run) uses S buffer u & 1 of the group, so the tensor core computes the scores of step u + 1
+        // while the group's softmax works on step u.
         if (lane == 0) {
             bool ok = true;
-            int gt = 0;               // KV tiles issued so far (all items): ring position
-            int cnt[2] = {0, 0};      // tiles handed to each softmax group so far: S/P phase
+            int gt = 0;               // KV tiles before this item (all items): ring position
+            int cnt0 = 0, cnt1 = 0;   // steps handed to each softmax group so far
             int item_no = 0;
             TItem it_next = load_titem(p, i0, i1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
                 it_next = load_titem(p, ii + 1, i1);      // in flight while this item runs
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
+                const bool dual = it.ntok * G > kTile;
                 ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
+                // the S buffers hold the previous item's softmax statistics until its epilogue is over
+                if (ok && item_no > 0) ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 27);
                 if (ok) tc_fence_after();
-                // S[b] <- Q K_j^T for tile j of the item (b = j & 1); S[b] is free once group b has turned
-                // its previous tile into P
+                int local0 = 0, local1 = 0;      // steps of this item issued to each group
                 for (int j = 0; j < ntiles && ok; ++j) {
-                    const int g = gt + j, b = j & 1;
-                    const int s = g % kKS;
-                    if (j >= 2)
-                        ok = mbar_wait(bar(kPFull0 + b), (uint32_t)(cnt[b] + (j >> 1) - 1) & 1u, abort_flag, p.status, 23);
-                    ok = ok && mbar_wait(bar(kKFull0 + s), (uint32_t)(g / kKS) & 1u, abort_flag, p.status, 21);
-                    if (!ok) break;
-                    tc_fence_after();
+                    const int pos = ring_pos_k(gt + j), s = pos % kRing;
+                    ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
                     const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                    const uint32_t idesc = instr_desc(16u * (uint32_t)npg, 0);
-                    const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
+                    for (int h = 0; h * 4 < npg && ok; ++h) {
+                        const uint32_t idesc = instr_desc(16u * (uint32_t)min(4, npg - 4 * h), 0);
+                        for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
+                            const int u = b ? cnt1 : cnt0, buf = u & 1;
+                            // the buffer (S, then P on top of it) is free once the P V of step u - 2 is done
+                            if ((b ? local1 : local0) >= 2)
+                                ok = mbar_wait(bar(kPvDone0 + 2 * b + buf), (uint32_t)((u >> 1) - 1) & 1u, abort_flag, p.status, 23);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t d = tmem + kColS + 128u * (uint32_t)b + 64u * (uint32_t)buf;
+                            const uint32_t qbase = sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u);
+                            const uint32_t kbase = sbase + kOffRing + s * kTileBytes + (uint32_t)h * (kSub * 128u);
 #pragma unroll
-                    for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        mma_f16(d, smem_desc(sbase + kOffQ + off, 16, 1024),
-                                smem_desc(sbase + kOffK + s * kTileBytes + off, 16, 1024), idesc, ks > 0);
+                            for (int ks = 0; ks < kD / 16; ++ks) {
+                                const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                                mma_f16(d, smem_desc(qbase + off, 16, 1024), smem_desc(kbase + off, 16, 1024), idesc, ks > 0);
+                            }
+                            mma_commit(bar(kSFull0 + 2 * b + buf));
+                            if (b) { ++cnt1; ++local1; } else { ++cnt0; ++local0; }
+                        }
                     }
-                    mma_commit(bar(kKEmpty0 + s));
-                    mma_commit(bar(kSFull0 + b));
+                    if (ok) mma_commit(bar(kRingEmpty0 + s));
                 }
                 gt += ntiles;
-                cnt[0] += (ntiles + 1) >> 1;
-                cnt[1] += ntiles >> 1;
             }
             // make sure nothing is still running on the tensor core before tensor memory is released
             mma_commit(bar(kMmaDrain));
@@ -359,7 +406,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         if (lane == 0) {
             bool ok = true;
             int gt = 0;
-            int cnt[2] = {0, 0};
+            int cnt0 = 0, cnt1 = 0;
             int item_no = 0;
             const uint32_t idesc_pv = instr_desc(128, 1);
             TItem it_next = load_titem(p, i0, i1);
@@ -367,31 +414,35 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 const TItem it = it_next;
                 it_next = load_titem(p, ii + 1, i1);
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
-                // O[b] (+)= P_j V_j: P[b] comes from group b, V from the ring; the first P V into each
-                // accumulator of an item overwrites it, so the previous item's epilogue must be done
+                const bool dual = it.ntok * G > kTile;
+                // O[b] (+)= P V: P (tensor memory) comes from group b, V from the ring; the first P V into
+                // an accumulator of an item overwrites it, so the previous item's epilogue must be done
+                if (item_no > 0) ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
+                int first0 = 1, first1 = 1;
                 for (int j = 0; j < ntiles && ok; ++j) {
-                    const int g = gt + j, b = j & 1;
-                    const int s = g % kVS;
-                    ok = mbar_wait(bar(kPFull0 + b), (uint32_t)(cnt[b] + (j >> 1)) & 1u, abort_flag, p.status, 26) &&
-                         mbar_wait(bar(kVFull0 + s), (uint32_t)(g / kVS) & 1u, abort_flag, p.status, 24);
-                    if (ok && j == 0 && item_no > 0)
-                        ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
-                    if (!ok) break;
-                    tc_fence_after();
+                    const int pos = ring_pos_v(gt + j), s = pos % kRing;
+                    ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
                     const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                    for (int ks = 0; ks < npg; ++ks) {
-                        const uint32_t poff = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        mma_f16(tmem + kColO + 128u * (uint32_t)b,
-                                smem_desc(sbase + kOffP + b * kTileBytes + poff, 16, 1024),
-                                smem_desc(sbase + kOffV + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
-                                idesc_pv, (j > 1 || ks > 0) ? 1u : 0u);
+                    for (int h = 0; h * 4 < npg && ok; ++h) {
+                        const int nk = min(4, npg - 4 * h);        // pages (K steps of 16 keys) in this step
+                        for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
+                            const int u = b ? cnt1 : cnt0, buf = u & 1;
+                            ok = mbar_wait(bar(kPFull0 + 2 * b + buf), (uint32_t)(u >> 1) & 1u, abort_flag, p.status, 26);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const bool fresh = b ? first1 : first0;
+                            const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b + 64u * (uint32_t)buf;
+                            for (int ks = 0; ks < nk; ++ks)
+                                mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks,
+                                           smem_desc(sbase + kOffRing + s * kTileBytes + (uint32_t)(4 * h + ks) * 2 * 1024u, kHalfBytes, 1024),
+                                           idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
+                            if (b) { first1 = 0; ++cnt1; } else { first0 = 0; ++cnt0; }
+                            mma_commit(bar(kPvDone0 + 2 * b + buf));
+                        }
                     }
-                    mma_commit(bar(kVEmpty0 + s));
-                    mma_commit(bar(kPvDone0 + b));
+                    if (ok) mma_commit(bar(kRingEmpty0 + s));
                 }
                 gt += ntiles;
-                cnt[0] += (ntiles + 1) >> 1;
-                cnt[1] += ntiles >> 1;
             }
             mma_commit(bar(kMmaDrain + 1));
             const long long t0 = clock64();
@@ -403,180 +454,207 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         if constexpr (FUSED) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxFused));
         // ------------------------------------------------------------------ softmax / epilogue groups
         const int b = warp >> 2;                   // softmax group
-        const int m = threadIdx.x & 127;           // query row of the tile = tensor-memory lane
-        const int t = m / G, g = m % G;
+        const int m = threadIdx.x & 127;           // row of the group's tile = tensor-memory lane
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        const uint32_t s_addr = lane_addr + kColS + 128u * (uint32_t)b;
+        const uint32_t s_addr = lane_addr + kColS + 128u * (uint32_t)b;      // + 64 * buffer
         const uint32_t o_addr = lane_addr + kColO + 128u * (uint32_t)b;
-        uint8_t* p_smem = smem + kOffP + b * kTileBytes;
-        // (max, sum) of each group and row for the epilogue live at the start of that group's P buffer:
-        // P[b] is idle from the group's last P.V until the next item's first Q K^T, which cannot be
-        // issued before every thread has read the statistics and staged the next Q.
-        float2* stats0 = reinterpret_cast<float2*>(smem + kOffP);
-        float2* stats1 = reinterpret_cast<float2*>(smem + kOffP + kTileBytes);
         const float qscale = p.sm_scale * kLog2e;
-        int gt = 0;          // KV tiles before this item (all groups)
-        int cnt = 0;         // tiles this group has processed before this item
+        const float2 qscale2 = make_float2(qscale, qscale);
+        int cnt = 0;         // steps this group has processed before this item
         int item_no = 0;
         bool ok = true;
-        // This thread's share of an item's Q: row m, the 8 chunks (16 bytes each) of value half b.  The
-        // next item's descriptor and Q rows are fetched while the current item runs.
-        auto load_q = [&](const TItem& x, uint4 (&w)[8]) {
-            const bool valid = x.kv_end > 0 && t < x.ntok;
+        // This thread's share of an item's Q.  Dual items: the whole row 128 b + m (16 chunks of 16
+        // bytes) into Q[b]; otherwise value half b of row m (8 chunks) into Q[0].  The next item's Q is
+        // fetched at the end of the current item's KV loop, ahead of the epilogue.
+        auto load_q = [&](const TItem& x, uint4 (&w)[16]) {
+            const bool dual = x.ntok * G > kTile;
+            const int r = dual ? 128 * b + m : m;
+            const bool valid = x.kv_end > 0 && r / G < x.ntok;
             const uint4* src = reinterpret_cast<const uint4*>(
-                q + ((size_t)(x.q_row0 + t) * Hq + (size_t)x.kv_head * G + g) * kD) + 8 * b;
+                q + ((size_t)(x.q_row0 + r / G) * Hq + (size_t)x.kv_head * G + r % G) * kD) + (dual ? 0 : 8 * b);
 #pragma unroll
             for (int c = 0; c < 8; ++c) w[c] = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int c = 8; c < 16; ++c) w[c] = (valid && dual) ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
         };
         TItem it_next = load_titem(p, i0, i1);
-        uint4 q_next[8];
+        uint4 q_next[16];
+        pdl_wait();
         load_q(it_next, q_next);
         for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
             const TItem it = it_next;
             const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
+            const bool dual = it.ntok * G > kTile;
+            const int r = dual ? 128 * b + m : m;      // query row of the item
+            const int t = r / G, g = r % G;
             const bool row_valid = t < it.ntok;
             // ---- stage Q with the 128-byte swizzle the MMA descriptor expects
+            if (dual) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4*>(smem + kOffQ + b * kHalfBytes + m * 128 + ((c ^ (m & 7)) << 4)) = q_next[c];
+                for (int c = 0; c < 16; ++c)
+                    *reinterpret_cast<uint4*>(smem + kOffQ + b * kTileBytes + (c >> 3) * kHalfBytes + m * 128 +
+                                              (((c & 7) ^ (m & 7)) << 4)) = q_next[c];
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4*>(smem + kOffQ + b * kHalfBytes + m * 128 + ((c ^ (m & 7)) << 4)) = q_next[c];
+            }
             fence_async_smem();
             mbar_arrive(bar(kQFull));
             it_next = load_titem(p, ii + 1, i1);
-            load_q(it_next, q_next);
             const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
-            float m_ref = -INFINITY, l_sum = 0.f;
-            int mine = 0;                                                          // tiles of this group so far
-            for (int j = b; j < ntiles && ok; j += 2, ++mine) {
-                const int base = it.kv0 + j * kTile;
-                const int vis = max(0, min(kTile, lim_row - base));     // visible columns of this row
-                ok = mbar_wait_warp(bar(kSFull0 + b), (uint32_t)(cnt + mine) & 1u, abort_flag, p.status, 31);
-                if (!ok) break;
-                tc_fence_after();
-                const bool full_tile = __all_sync(0xffffffffu, vis == kTile);
-                if (mine == 0) {
-                    // first tile of the group: the reference maximum is this tile's row maximum
-                    float tmax = -INFINITY;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(s_addr + 32u * c, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            tmax = fmaxf(tmax, (full_tile || c * 32 + e < vis) ? __uint_as_float(r[e]) : -INFINITY);
-                    }
-                    m_ref = tmax * qscale;     // qscale > 0: the maximum commutes with the scaling
-                } else {
-                    // P[b] and O[b] are still in use by the P.V of this group's previous tile
-                    ok = mbar_wait_warp(bar(kPvDone0 + b), (uint32_t)(cnt + mine - 1) & 1u, abort_flag, p.status, 32);
+            float m_ref = -INFINITY;                     // reference maximum (log2 domain)
+            float2 l2 = make_float2(0.f, 0.f);           // running sum of P, two partial sums
+            int mine = 0;                                // steps of this group so far in this item
+            for (int j = dual ? 0 : b; j < ntiles && ok; j += dual ? 1 : 2) {
+                const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
+                for (int h = 0; h * 4 < npg && ok; ++h, ++mine) {
+                    const int u = cnt + mine, buf = u & 1;
+                    const int base = it.kv0 + j * kTile + h * kSub;
+                    const int vis = max(0, min(kSub, lim_row - base));      // visible columns of this row
+                    const uint32_t sb = s_addr + 64u * (uint32_t)buf;
+                    ok = mbar_wait_warp(bar(kSFull0 + 2 * b + buf), (uint32_t)(u >> 1) & 1u, abort_flag, p.status, 31);
                     if (!ok) break;
                     tc_fence_after();
-                }
-                // P = exp2(S * scale - m_ref) as bf16 into shared memory (A operand of P.V).  The
-                // reference maximum is only moved when some score exceeds it by the threshold; then O[b]
-                // and the running sum are rescaled and the tile is redone.
-                float l_tile = 0.f;
-#pragma unroll 1
-                for (int attempt = 0; attempt < 2; ++attempt) {
+                    uint32_t rr[64];
+                    tmem_ld32(sb, *reinterpret_cast<uint32_t(*)[32]>(&rr[0]));
+                    tmem_ld32(sb + 32u, *reinterpret_cast<uint32_t(*)[32]>(&rr[32]));
+                    tmem_wait_ld();
+                    // x = S * scale - m_ref (log2 domain), two values per instruction
                     const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-                    float tmax = -INFINITY;
-                    l_tile = 0.f;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(s_addr + 32u * c, r);
-                        tmem_wait_ld();
-                        uint32_t pk[16];
+                    const float2 nm2 = make_float2(-m_use, -m_use);
+                    float2 x[32];
 #pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            float s0 = __uint_as_float(r[e]), s1 = __uint_as_float(r[e + 1]);
-                            if (!full_tile) {
-                                if (c * 32 + e >= vis) s0 = -INFINITY;
-                                if (c * 32 + e + 1 >= vis) s1 = -INFINITY;
+                    for (int e = 0; e < 32; ++e)
+                        x[e] = __ffma2_rn(make_float2(__uint_as_float(rr[2 * e]), __uint_as_float(rr[2 * e + 1])), qscale2, nm2);
+                    if (!__all_sync(0xffffffffu, vis == kSub)) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            if (2 * e >= vis) x[e].x = -INFINITY;
+                            if (2 * e + 1 >= vis) x[e].y = -INFINITY;
+                        }
+                    }
+                    auto xv = [&](int k) { return (k & 1) ? x[k >> 1].y : x[k >> 1].x; };
+                    float cmax = fmax3(xv(0), xv(1), xv(2));
+#pragma unroll
+                    for (int k = 3; k < 63; k += 2) cmax = fmax3(cmax, xv(k), xv(k + 1));
+                    cmax = fmaxf(cmax, xv(63));
+                    // x is relative to m_ref (to 0 while the row has no reference yet: then any visible key sets it)
+                    if (__any_sync(0xffffffffu, cmax > (m_ref == -INFINITY ? -INFINITY : kRescaleThreshold))) {
+                        // Move the reference maximum (rare after the first step): rescale the running sum
+                        // and, once the P V of the previous step has landed, O[b]; shift this step's x.
+                        const float m_new = cmax == -INFINITY ? m_ref : fmaxf(m_ref, m_use + cmax);
+                        const float scale = m_new == -INFINITY ? 1.f : fast_exp2(m_ref - m_new);
+                        const float shift = (m_new == -INFINITY ? 0.f : m_new) - m_use;
+                        m_ref = m_new;
+                        l2.x *= scale;
+                        l2.y *= scale;
+                        const float2 ns2 = make_float2(-shift, -shift);
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) x[e] = __fadd2_rn(x[e], ns2);
+                        if (mine > 0) {
+                            ok = mbar_wait_warp(bar(kPvDone0 + 2 * b + (buf ^ 1)), (uint32_t)((u - 1) >> 1) & 1u, abort_flag, p.status, 32);
+                            if (!ok) break;
+                            tc_fence_after();
+#pragma unroll 1
+                            for (int cc = 0; cc < 8; ++cc) {
+                                uint32_t ro[16];
+                                tmem_ld16(o_addr + 16u * cc, ro);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) ro[e] = __float_as_uint(__uint_as_float(ro[e]) * scale);
+                                tmem_st16(o_addr + 16u * cc, ro);
                             }
-                            tmax = fmaxf(tmax, fmaxf(s0, s1));
-                            const float p0 = fast_exp2(fmaf(s0, qscale, -m_use));
-                            const float p1 = fast_exp2(fmaf(s1, qscale, -m_use));
-                            l_tile += p0 + p1;
-                            pk[e >> 1] = pack_bf16x2(p0, p1);
-                        }
-                        // columns [32c, 32c+32) = 4 chunks of 8 keys: key half c >> 1, chunks (c & 1) * 4 ..
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const int cc = (c & 1) * 4 + k;
-                            *reinterpret_cast<uint4*>(p_smem + (c >> 1) * kHalfBytes + m * 128 + ((cc ^ (m & 7)) << 4)) =
-                                make_uint4(pk[4 * k], pk[4 * k + 1], pk[4 * k + 2], pk[4 * k + 3]);
+                            tmem_wait_st();
                         }
                     }
-                    tmax *= qscale;
-                    if (attempt == 1 || !__any_sync(0xffffffffu, tmax > m_ref + kRescaleThreshold)) break;
-                    const float m_new = fmaxf(m_ref, tmax);
-                    const float scale = m_new == -INFINITY ? 1.f : fast_exp2(m_ref - m_new);
-                    m_ref = m_new;
-                    l_sum *= scale;
-#pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(o_addr + 32u * c, r);
-                        tmem_wait_ld();
+                    // P = exp2(x) as packed bf16 over the first 32 columns of the buffer
+                    uint32_t pk[32];
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * scale);
-                        tmem_st32(o_addr + 32u * c, r);
+                    for (int e = 0; e < 32; ++e) {
+                        const float2 pe = make_float2(fast_exp2(x[e].x), fast_exp2(x[e].y));
+                        l2 = __fadd2_rn(l2, pe);
+                        pk[e] = pack_bf16x2(pe.x, pe.y);
                     }
+                    tmem_st16(sb, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
+                    tmem_st16(sb + 16u, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
                     tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar(kPFull0 + 2 * b + buf));
                 }
-                l_sum += l_tile;
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(bar(kPFull0 + b));
             }
             if (!ok) break;
-            // ---- epilogue: merge the two groups' states, group b writes value half b of every row
+            const float l_sum = l2.x + l2.y;
+            load_q(it_next, q_next);        // in flight during the epilogue
+            // ---- epilogue.  The groups' (max, sum) go through columns 0-1 of their first S buffer; the S
+            // buffers are idle from the group's last P V until the next item's first Q K^T.
             if (mine > 0) {
-                ok = mbar_wait_warp(bar(kPvDone0 + b), (uint32_t)(cnt + mine - 1) & 1u, abort_flag, p.status, 34);
+                const int ul = cnt + mine - 1;
+                ok = mbar_wait_warp(bar(kPvDone0 + 2 * b + (ul & 1)), (uint32_t)(ul >> 1) & 1u, abort_flag, p.status, 34);
                 if (!ok) break;
                 tc_fence_after();
             }
-            (b == 0 ? stats0 : stats1)[m] = make_float2(m_ref, l_sum);
+            tmem_st2(s_addr, __float_as_uint(m_ref), __float_as_uint(l_sum));
+            tmem_wait_st();
+            tc_fence_before();
             mbar_arrive(bar(kStats));
             ok = mbar_wait_warp(bar(kStats), (uint32_t)item_no & 1u, abort_flag, p.status, 35);
             if (!ok) break;
-            const float2 st0 = stats0[m], st1 = stats1[m];
-            const float M = fmaxf(st0.x, st1.x);
-            const float a0 = st0.y > 0.f ? fast_exp2(st0.x - M) : 0.f;
-            const float a1 = st1.y > 0.f ? fast_exp2(st1.x - M) : 0.f;
-            const float L = a0 * st0.y + a1 * st1.y;
-            const float inv = L > 0.f ? 1.f / L : 0.f;
-            const float w0 = a0 * inv, w1 = a1 * inv;
-            const float lse2 = L > 0.f ? M + log2f(L) : -INFINITY;
+            tc_fence_after();
             const size_t hq = (size_t)it.kv_head * G + g;
-            const size_t prow = it.partial_base < 0 ? 0 : (size_t)it.partial_base + (size_t)it.chunk * it.ntok + t;
+            const size_t prow = it.partial_row0 < 0 ? 0 : (size_t)it.partial_row0 + t;
+            float w0, w1, lse2;          // weights of O[0] and O[1] in this thread's output row
+            int c_begin, c_end;          // 32-column chunks of the row this thread writes
+            if (dual) {
+                const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+                w0 = b == 0 ? inv : 0.f;
+                w1 = b == 1 ? inv : 0.f;
+                lse2 = l_sum > 0.f ? m_ref + log2f(l_sum) : -INFINITY;
+                c_begin = 0; c_end = 4;
+            } else {
+                // the two groups hold two KV splits of the same rows: merge them; group b writes value half b
+                uint32_t x0, y0, x1, y1;
+                tmem_ld2(lane_addr + kColS, x0, y0);
+                tmem_ld2(lane_addr + kColS + 128u, x1, y1);
+                tmem_wait_ld();
+                const float m0 = __uint_as_float(x0), l0 = __uint_as_float(y0);
+                const float m1 = __uint_as_float(x1), l1 = __uint_as_float(y1);
+                const float M = fmaxf(m0, m1);
+                const float a0 = l0 > 0.f ? fast_exp2(m0 - M) : 0.f;
+                const float a1 = l1 > 0.f ? fast_exp2(m1 - M) : 0.f;
+                const float L = a0 * l0 + a1 * l1;
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+                w0 = a0 * inv;
+                w1 = a1 * inv;
+                lse2 = L > 0.f ? M + log2f(L) : -INFINITY;
+                c_begin = 2 * b; c_end = 2 * b + 2;
+            }
             const bool use0 = __any_sync(0xffffffffu, w0 != 0.f), use1 = __any_sync(0xffffffffu, w1 != 0.f);
 #pragma unroll 1
-            for (int c = 2 * b; c < 2 * b + 2; ++c) {
+            for (int c = c_begin; c < c_end; ++c) {
                 float acc[32];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) acc[e] = 0.f;
                 if (use0) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_addr + kColO + 32u * c, r);
+                    uint32_t ro[32];
+                    tmem_ld32(lane_addr + kColO + 32u * c, ro);
                     tmem_wait_ld();
                     if (w0 != 0.f) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) acc[e] = __uint_as_float(r[e]) * w0;
+                        for (int e = 0; e < 32; ++e) acc[e] = __uint_as_float(ro[e]) * w0;
                     }
                 }
                 if (use1) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_addr + kColO + 128u + 32u * c, r);
+                    uint32_t ro[32];
+                    tmem_ld32(lane_addr + kColO + 128u + 32u * c, ro);
                     tmem_wait_ld();
                     if (w1 != 0.f) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) acc[e] = fmaf(__uint_as_float(r[e]), w1, acc[e]);
+                        for (int e = 0; e < 32; ++e) acc[e] = fmaf(__uint_as_float(ro[e]), w1, acc[e]);
                     }
                 }
                 if (row_valid) {
-                    if (it.partial_base < 0) {
+                    if (it.partial_row0 < 0) {
                         uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(it.q_row0 + t) * Hq + hq) * kD + c * 32);
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
@@ -590,8 +668,8 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     }
                 }
             }
-            if (row_valid && b == 0) {
-                if (it.partial_base < 0) {
+            if (row_valid && (dual || b == 0)) {
+                if (it.partial_row0 < 0) {
                     if (lse != nullptr) lse[(size_t)(it.q_row0 + t) * Hq + hq] = lse2 * kLn2;
                 } else {
                     p.partial_lse[prow * G + g] = lse2;
@@ -599,7 +677,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             }
             tc_fence_before();
             mbar_arrive(bar(kOFree));
-            gt += ntiles;
             cnt += mine;
         }
     }

@@ -219,14 +219,10 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         auto load_item = [&](int ii) {
             PItem r{0, 0, 0, 0, -1, 0};
             if (ii < i1) {
-                const Item it = p.items[ii];
-                const Unit u = p.units[it.unit];
-                r.kv0 = it.kv0;
-                r.kv_end = min(it.kv1, u.kv_limit0);
-                r.q_row0 = u.q_row0;
-                r.kv_head = u.kv_head;
-                r.partial_row = u.partial_base < 0 ? -1 : u.partial_base + it.chunk;
-                r.page0 = u.page_base + it.kv0 / kPage;
+                const int4* src = reinterpret_cast<const int4*>(p.works + ii);
+                const int4 a = __ldg(src), b = __ldg(src + 1);
+                r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z;
+                r.kv_head = b.y; r.partial_row = b.z; r.page0 = b.w;
             }
             return r;
         };

@@ -29,6 +29,7 @@ attn_decode_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const 
                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
     extern __shared__ uint8_t smem_raw[];
     pdl_wait();
+    pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
     dec::decode_body<D, G, false>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw));
 }
 
@@ -37,6 +38,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
 attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ pool,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ uint8_t smem_raw[];
+    pdl_trigger();      // the kernel behind this one may start its prologue; it waits for this grid to complete
     tc::tc_body<G, false>(p, q, pool, out, lse, aligned_smem(smem_raw));
 }
 
@@ -47,6 +49,7 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
                   int S) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = aligned_smem(smem_raw);
+    pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
     tc::tc_body<G, true>(p, q, pool, out, lse, smem);
     __syncthreads();      // tensor memory released, shared memory free for the second phase
     dec::decode_body<tc::kD, G, true>(p, &kv_map, q, out, lse, S, smem);

@@ -14,9 +14,11 @@ lse_merge_kernel(DevPlan p, __nv_bfloat16* __restrict__ out, float* __restrict__
     constexpr int EPL = D / 32;   // output elements per lane
     const int lane = threadIdx.x & 31;
     const int G = p.group;
+    // the plan was uploaded before the attention kernel started: read it while that kernel drains
     const int entry = p.merge_blocks[blockIdx.x];
-    const Unit u = p.units[entry >> 5];
-    const int pair = (entry & 31) * 4 + (threadIdx.x >> 5);
+    const Unit u = p.units[entry >> 6];
+    pdl_wait();     // the partial results are complete and visible from here on
+    const int pair = (entry & 63) * 4 + (threadIdx.x >> 5);
     if (pair >= u.ntok * G) return;
     const int t = pair / G, g = pair % G;
     const int n = u.n_chunks;
@@ -70,11 +72,13 @@ lse_merge_kernel(DevPlan p, __nv_bfloat16* __restrict__ out, float* __restrict__
 
 cudaError_t launch_lse_merge(const DevPlan& p, void* out, float* lse, cudaStream_t stream) {
     if (p.num_merge_blocks == 0) return cudaSuccess;
+    // Programmatic serialization: the attention kernels let their dependents start as soon as all of
+    // their CTAs are running, so this grid's launch and plan reads overlap the attention tail.
     if (p.head_dim == 128)
-        lse_merge_kernel<128><<<p.num_merge_blocks, 128, 0, stream>>>(p, (__nv_bfloat16*)out, lse);
-    else
-        lse_merge_kernel<64><<<p.num_merge_blocks, 128, 0, stream>>>(p, (__nv_bfloat16*)out, lse);
-    return cudaGetLastError();
+        return launch_pdl(lse_merge_kernel<128>, dim3(p.num_merge_blocks), dim3(128), 0, stream, p,
+                          (__nv_bfloat16*)out, lse);
+    return launch_pdl(lse_merge_kernel<64>, dim3(p.num_merge_blocks), dim3(128), 0, stream, p,
+                      (__nv_bfloat16*)out, lse);
 }
 
 }  // namespace asynclm

@@ -41,14 +41,15 @@ static int check_shape(const asynclm_shape* s) {
     return ASYNCLM_OK;
 }
 
-int tensor_tile_tokens(int group) { return 128 / group; }
+// Tokens of a span that one tensor-core work item covers: two row tiles of 128 (token, head) rows.
+int tensor_tile_tokens(int group) { return 256 / group; }
 
 static int default_tensor_min_rows() { return 32; }
 
 // Sizes of the sections of the packed blob (identical offsets on host and device).
 struct BlobLayout {
     size_t off_q_indptr, off_kv_len, off_page_indptr, off_page_indices, off_row_seq, off_units,
-        off_items, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
+        off_items, off_works, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
 };
 
 static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64_t n_units,
@@ -65,6 +66,7 @@ static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64
     L.off_row_seq = take(sizeof(int32_t) * (size_t)std::max(total_q, 1));
     L.off_units = take(sizeof(Unit) * (size_t)std::max<int64_t>(n_units, 1));
     L.off_items = take(sizeof(Item) * (size_t)std::max<int64_t>(n_items, 1));
+    L.off_works = take(sizeof(Work) * (size_t)std::max<int64_t>(n_items, 1));
     L.off_cta_cuda = take(sizeof(int32_t) * (size_t)(ctas_cuda + 1));
     L.off_cta_tensor = take(sizeof(int32_t) * (size_t)(ctas_tensor + 1));
     L.off_split = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_split, 1));
@@ -214,8 +216,9 @@ struct PathCost {
     int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
 };
 // (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
-constexpr PathCost kTensorCost{128, 1590, 4500, 4800};
+constexpr PathCost kTensorCost{128, 1500, 4000, 3000};
 constexpr PathCost kCudaCost{96, 1260, 1100, 6000};
+constexpr int64_t kTensorDualTileNs = 1900;   // a KV tile of an item with two row tiles (more than 128 rows)
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
 // then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
@@ -223,7 +226,7 @@ constexpr PathCost kCudaCost{96, 1260, 1100, 6000};
 // piece boundary falls inside it, so there are at most n_ctas - 1 more items than units, most CTAs
 // run one kind of work only, and the two kinds finish together.
 void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& ids_cuda,
-                  std::vector<UnitBuild>& units, int n_ctas, std::vector<Item>& items,
+                  std::vector<UnitBuild>& units, int group, int n_ctas, std::vector<Item>& items,
                   std::vector<int32_t>& cta_indptr_cuda, std::vector<int32_t>& cta_indptr_tensor,
                   std::vector<int32_t>& item_cta) {
     struct Piece { Item it; int32_t cta; };
@@ -231,10 +234,13 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     int64_t best_max = -1;
     const std::vector<int>* ids[2] = {&ids_tensor, &ids_cuda};
     const PathCost cost[2] = {kTensorCost, kCudaCost};
+    auto tile_ns = [&](int path, int id) {
+        return path == 0 && units[id].u.ntok * group > 128 ? kTensorDualTileNs : cost[path].tile_ns;
+    };
     int64_t total = 0;
     for (int path = 0; path < 2; ++path)
         for (int id : *ids[path])
-            total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * cost[path].tile_ns;
+            total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * tile_ns(path, id);
     total += (int64_t)n_ctas * (kTensorCost.item_ns + kCudaCost.phase_ns) / 2;
     int64_t quota = std::max<int64_t>(1, (total + n_ctas - 1) / n_ctas);
     for (int round = 0; round < 8; ++round) {
@@ -245,8 +251,9 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
         bool has_phase[2] = {false, false};
         auto next_cta = [&]() { ++cta; has_phase[0] = has_phase[1] = false; };
         for (int path = 0; path < 2; ++path) {
-            const PathCost& pc = cost[path];
+            PathCost pc = cost[path];
             for (int id : *ids[path]) {
+                pc.tile_ns = tile_ns(path, id);
                 int64_t left = (units[id].n_keys + pc.gran - 1) / pc.gran;   // tiles left
                 int64_t k0 = 0;
                 int c = 0;
@@ -438,7 +445,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
         cut_and_deal(ids_tensor, units, fixed_chunk, ctas_tensor, kTensorItemOverheadTiles, items,
                      cta_indptr_tensor, item_cta);
     } else {
-        deal_jointly(ids_tensor, ids_cuda, units, ctas_cuda, items, cta_indptr_cuda, cta_indptr_tensor, item_cta);
+        deal_jointly(ids_tensor, ids_cuda, units, G, ctas_cuda, items, cta_indptr_cuda, cta_indptr_tensor, item_cta);
         n_items_cuda = cta_indptr_cuda[(size_t)ctas_cuda];
     }
     const int n_items = (int)items.size();
@@ -451,8 +458,8 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
             units[i].u.partial_base = (int32_t)partial_rows;
             partial_rows += (int64_t)units[i].u.n_chunks * units[i].u.ntok;
             split_units.push_back((int32_t)i);
-            if (i >= (size_t)(INT32_MAX >> 5)) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
-            for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 5) | (size_t)rb));
+            if (i >= (size_t)(INT32_MAX >> 6)) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
+            for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
             if (partial_rows > INT32_MAX / 2) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
         }
     }
@@ -487,6 +494,21 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     Unit* h_units = (Unit*)(hb + L.off_units);
     for (size_t i = 0; i < units.size(); ++i) h_units[i] = units[i].u;
     if (n_items > 0) std::memcpy(hb + L.off_items, items.data(), sizeof(Item) * (size_t)n_items);
+    Work* h_works = (Work*)(hb + L.off_works);
+    for (int i = 0; i < n_items; ++i) {
+        const Item& it = items[(size_t)i];
+        const Unit& u = units[(size_t)it.unit].u;
+        Work w;
+        w.kv0 = it.kv0;
+        w.kv_end = std::min(it.kv1, u.kv_limit0 + u.ntok - 1);
+        w.q_row0 = u.q_row0;
+        w.ntok = u.ntok;
+        w.kv_limit0 = u.kv_limit0;
+        w.kv_head = u.kv_head;
+        w.partial_row0 = u.partial_base < 0 ? -1 : u.partial_base + it.chunk * u.ntok;
+        w.page0 = u.page_base + it.kv0 / kPage;
+        h_works[i] = w;
+    }
     std::memcpy(hb + L.off_cta_cuda, cta_indptr_cuda.data(), sizeof(int32_t) * (size_t)(ctas_cuda + 1));
     std::memcpy(hb + L.off_cta_tensor, cta_indptr_tensor.data(),
                 sizeof(int32_t) * (size_t)(ctas_tensor + 1));
@@ -519,6 +541,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     d.row_seq = (const int32_t*)dp(L.off_row_seq);
     d.units = (const Unit*)dp(L.off_units);
     d.items = (const Item*)dp(L.off_items);
+    d.works = (const Work*)dp(L.off_works);
     d.cta_indptr_cuda = (const int32_t*)dp(L.off_cta_cuda);
     d.cta_indptr_tensor = (const int32_t*)dp(L.off_cta_tensor);
     d.split_units = (const int32_t*)dp(L.off_split);

@@ -31,6 +31,19 @@ struct Item {
     int32_t chunk;         // chunk index inside the unit
 };
 
+// What an attention kernel needs to run one item, resolved by the planner so that a CTA reaches its
+// first page ids with two dependent loads (its item range, then this record).
+struct alignas(16) Work {
+    int32_t kv0;           // first key position
+    int32_t kv_end;        // one past the last key any token of the unit sees in this item
+    int32_t q_row0;        // global token row of the unit's first token
+    int32_t ntok;
+    int32_t kv_limit0;     // token t of the unit sees keys [0, kv_limit0 + t)
+    int32_t kv_head;
+    int32_t partial_row0;  // partial row of token 0 in this chunk; -1: the item writes final output
+    int32_t page0;         // index into page_indices of the page that holds key kv0
+};
+
 // Pointers into the device workspace, passed to kernels by value.
 struct DevPlan {
     const int32_t* q_indptr;
@@ -40,10 +53,11 @@ struct DevPlan {
     const int32_t* row_seq;          // [T] sequence of each new token row
     const Unit* units;
     const Item* items;               // CUDA-core items first (grouped by CTA), then tensor items
+    const Work* works;               // [num_items] the same items, resolved for the kernels
     const int32_t* cta_indptr_cuda;  // [num_ctas_cuda + 1] into items
     const int32_t* cta_indptr_tensor;// [num_ctas_tensor + 1] into items (absolute indices)
     const int32_t* split_units;      // [num_split_units] unit ids that need a merge
-    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 5) | row block: 4 (token, head) rows each
+    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 6) | row block: 4 (token, head) rows each
     float* partial_o;                // [partial_rows][G][d]
     float* partial_lse;              // [partial_rows][G]   (log2 domain)
     int32_t* status;                 // device status word
