@@ -44,7 +44,7 @@ constexpr int kThreads = 384;
 constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10, kMmaWarpPV = 11;
 constexpr int kD = 128;
 constexpr int kTile = 128;                       // keys per K/V ring slot and query rows per row tile
-constexpr int kSub = 64;                         // keys per softmax step (one S buffer)
+constexpr int kSub = 64;                         // keys the softmax handles at a time (half an S tile)
 constexpr int kRing = 5;                         // K/V ring slots
 constexpr uint32_t kHalfBytes = 128 * 128;       // one 64-value half of a 128-row tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;  // 32 KiB
@@ -55,7 +55,7 @@ constexpr long long kWaitCycles = 2000000000ll;
 constexpr uint32_t kOffQ = 0;                           // Q[0], Q[1]
 constexpr uint32_t kOffRing = kOffQ + 2 * kTileBytes;
 constexpr uint32_t kOffBar = kOffRing + kRing * kTileBytes;
-// S, P V and P hand-offs exist per (group b, S buffer): index 2 * b + buffer
+// S, P V and P hand-offs exist per group b: index 2 * b
 enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPvDone0 = kPFull0 + 4, kSFull0 = kPvDone0 + 4,
            kRingFull0 = kSFull0 + 4, kRingEmpty0 = kRingFull0 + kRing, kMmaDrain = kRingEmpty0 + kRing,
            kMmaDrain2, kNumBars };
@@ -65,8 +65,7 @@ constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
 // tensor memory columns
-constexpr uint32_t kColS = 0;      // group b: two S buffers of 64 columns each at 128 b + 64 buffer; the P of a
-                                   // buffer overlays its first 32 columns
+constexpr uint32_t kColS = 0;      // S[0], S[1]: 128 columns each; P[b] overlays the first 64 of S[b]
 constexpr uint32_t kColO = 256;    // O[0], O[1]: 128 columns each
 constexpr uint32_t kTmemCols = 512;
 
@@ -219,10 +218,11 @@ struct TItem {
     int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row0, page0;
 };
 
-__device__ __forceinline__ TItem load_titem(const DevPlan& p, int ii, int i1) {
+// `rec`: a Work record (the planner's array, or the copy of a CTA's first item in its header).
+__device__ __forceinline__ TItem load_titem(const Work* rec, bool valid) {
     TItem r{0, 0, 0, 0, 0, 0, -1, 0};
-    if (ii < i1) {
-        const int4* src = reinterpret_cast<const int4*>(p.works + ii);
+    if (valid) {
+        const int4* src = reinterpret_cast<const int4*>(rec);
         const int4 a = __ldg(src), b = __ldg(src + 1);
         r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z; r.ntok = a.w;
         r.kv_limit0 = b.x; r.kv_head = b.y; r.partial_row0 = b.z; r.page0 = b.w;
@@ -253,7 +253,9 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
     const int Hq = p.num_q_heads, Hkv = p.num_kv_heads;
     // The plan was uploaded before the kernel in front of this one started, so it may be read before
     // pdl_wait(); everything else (pool, q, outputs) is touched only after it.
-    const int i0 = p.cta_indptr_tensor[blockIdx.x], i1 = p.cta_indptr_tensor[blockIdx.x + 1];
+    const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
+    const int i0 = head[0], i1 = head[1];
+    const Work* head_work = reinterpret_cast<const Work*>(head + kHeadWorkTensor);      // = p.works[i0]
 
     if (threadIdx.x == 0) {
         mbar_init(bar(kQFull), 256);
@@ -299,11 +301,11 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         bool ok = true;
         int n = 0;                                             // KV tiles issued so far (all items)
         int last_pos = -1;
-        TItem cur = load_titem(p, i0, i1), nxt = load_titem(p, i0 + 1, i1);
-        int pages_cur = cur.kv_end > 0 ? load_pages(cur, 0) : 0;
+        TItem cur = load_titem(head_work, i0 < i1), nxt = load_titem(p.works + i0 + 1, i0 + 1 < i1);
+        int pages_cur = head[kHeadPagesTensor + lane];      // the first item's first 32 page ids (0 beyond its end)
         pdl_wait();
         for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
-            const TItem after = load_titem(p, ii + 2, i1);
+            const TItem after = load_titem(p.works + ii + 2, ii + 2 < i1);
             const int ntiles = (cur.kv_end - cur.kv0 + kTile - 1) / kTile;
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
@@ -347,49 +349,46 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ Q K^T issuer
-        // A KV tile is consumed in steps of 64 keys.  Step u of group b (counted over the CTA's whole
-        // run) uses S buffer u & 1 of the group, so the tensor core computes the scores of step u + 1
-        // while the group's softmax works on step u.
+        // An MMA costs about 94 cycles however narrow it is (measured), so Q K^T is issued 128 keys wide:
+        // 8 instructions per tile and group.
         if (lane == 0) {
             bool ok = true;
             int gt = 0;               // KV tiles before this item (all items): ring position
             int cnt0 = 0, cnt1 = 0;   // steps handed to each softmax group so far
             int item_no = 0;
-            TItem it_next = load_titem(p, i0, i1);
+            TItem it_next = load_titem(head_work, i0 < i1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
-                it_next = load_titem(p, ii + 1, i1);      // in flight while this item runs
+                it_next = load_titem(p.works + ii + 1, ii + 1 < i1);      // in flight while this item runs
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
                 const bool dual = it.ntok * G > kTile;
                 ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
                 // the S buffers hold the previous item's softmax statistics until its epilogue is over
                 if (ok && item_no > 0) ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 27);
                 if (ok) tc_fence_after();
-                int local0 = 0, local1 = 0;      // steps of this item issued to each group
+                int local0 = 0, local1 = 0;      // tiles of this item issued to each group
                 for (int j = 0; j < ntiles && ok; ++j) {
                     const int pos = ring_pos_k(gt + j), s = pos % kRing;
                     ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
                     const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                    for (int h = 0; h * 4 < npg && ok; ++h) {
-                        const uint32_t idesc = instr_desc(16u * (uint32_t)min(4, npg - 4 * h), 0);
-                        for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
-                            const int u = b ? cnt1 : cnt0, buf = u & 1;
-                            // the buffer (S, then P on top of it) is free once the P V of step u - 2 is done
-                            if ((b ? local1 : local0) >= 2)
-                                ok = mbar_wait(bar(kPvDone0 + 2 * b + buf), (uint32_t)((u >> 1) - 1) & 1u, abort_flag, p.status, 23);
-                            if (!ok) break;
-                            tc_fence_after();
-                            const uint32_t d = tmem + kColS + 128u * (uint32_t)b + 64u * (uint32_t)buf;
-                            const uint32_t qbase = sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u);
-                            const uint32_t kbase = sbase + kOffRing + s * kTileBytes + (uint32_t)h * (kSub * 128u);
+                    const uint32_t idesc = instr_desc(16u * (uint32_t)npg, 0);
+                    for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
+                        const int u = b ? cnt1 : cnt0;
+                        // S[b] (and P[b] on top of it) is free once the P V of the group's previous tile is done
+                        if ((b ? local1 : local0) >= 1)
+                            ok = mbar_wait(bar(kPvDone0 + 2 * b), (uint32_t)(u - 1) & 1u, abort_flag, p.status, 23);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
+                        const uint32_t qbase = sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u);
+                        const uint32_t kbase = sbase + kOffRing + s * kTileBytes;
 #pragma unroll
-                            for (int ks = 0; ks < kD / 16; ++ks) {
-                                const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                                mma_f16(d, smem_desc(qbase + off, 16, 1024), smem_desc(kbase + off, 16, 1024), idesc, ks > 0);
-                            }
-                            mma_commit(bar(kSFull0 + 2 * b + buf));
-                            if (b) { ++cnt1; ++local1; } else { ++cnt0; ++local0; }
+                        for (int ks = 0; ks < kD / 16; ++ks) {
+                            const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                            mma_f16(d, smem_desc(qbase + off, 16, 1024), smem_desc(kbase + off, 16, 1024), idesc, ks > 0);
                         }
+                        mma_commit(bar(kSFull0 + 2 * b));
+                        if (b) { ++cnt1; ++local1; } else { ++cnt0; ++local0; }
                     }
                     if (ok) mma_commit(bar(kRingEmpty0 + s));
                 }
@@ -409,10 +408,10 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             int cnt0 = 0, cnt1 = 0;
             int item_no = 0;
             const uint32_t idesc_pv = instr_desc(128, 1);
-            TItem it_next = load_titem(p, i0, i1);
+            TItem it_next = load_titem(head_work, i0 < i1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
-                it_next = load_titem(p, ii + 1, i1);
+                it_next = load_titem(p.works + ii + 1, ii + 1 < i1);
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
                 const bool dual = it.ntok * G > kTile;
                 // O[b] (+)= P V: P (tensor memory) comes from group b, V from the ring; the first P V into
@@ -423,22 +422,19 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     const int pos = ring_pos_v(gt + j), s = pos % kRing;
                     ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
                     const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                    for (int h = 0; h * 4 < npg && ok; ++h) {
-                        const int nk = min(4, npg - 4 * h);        // pages (K steps of 16 keys) in this step
-                        for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
-                            const int u = b ? cnt1 : cnt0, buf = u & 1;
-                            ok = mbar_wait(bar(kPFull0 + 2 * b + buf), (uint32_t)(u >> 1) & 1u, abort_flag, p.status, 26);
-                            if (!ok) break;
-                            tc_fence_after();
-                            const bool fresh = b ? first1 : first0;
-                            const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b + 64u * (uint32_t)buf;
-                            for (int ks = 0; ks < nk; ++ks)
-                                mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks,
-                                           smem_desc(sbase + kOffRing + s * kTileBytes + (uint32_t)(4 * h + ks) * 2 * 1024u, kHalfBytes, 1024),
-                                           idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
-                            if (b) { first1 = 0; ++cnt1; } else { first0 = 0; ++cnt0; }
-                            mma_commit(bar(kPvDone0 + 2 * b + buf));
-                        }
+                    for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
+                        const int u = b ? cnt1 : cnt0;
+                        ok = mbar_wait(bar(kPFull0 + 2 * b), (uint32_t)u & 1u, abort_flag, p.status, 26);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const bool fresh = b ? first1 : first0;
+                        const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b;
+                        for (int ks = 0; ks < npg; ++ks)
+                            mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks,
+                                       smem_desc(sbase + kOffRing + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
+                                       idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
+                        if (b) { first1 = 0; ++cnt1; } else { first0 = 0; ++cnt0; }
+                        mma_commit(bar(kPvDone0 + 2 * b));
                     }
                     if (ok) mma_commit(bar(kRingEmpty0 + s));
                 }
@@ -460,7 +456,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         const uint32_t o_addr = lane_addr + kColO + 128u * (uint32_t)b;
         const float qscale = p.sm_scale * kLog2e;
         const float2 qscale2 = make_float2(qscale, qscale);
-        int cnt = 0;         // steps this group has processed before this item
+        int cnt = 0;         // tiles this group has processed before this item
         int item_no = 0;
         bool ok = true;
         // This thread's share of an item's Q.  Dual items: the whole row 128 b + m (16 chunks of 16
@@ -477,7 +473,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
 #pragma unroll
             for (int c = 8; c < 16; ++c) w[c] = (valid && dual) ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
         };
-        TItem it_next = load_titem(p, i0, i1);
+        TItem it_next = load_titem(head_work, i0 < i1);
         uint4 q_next[16];
         pdl_wait();
         load_q(it_next, q_next);
@@ -488,7 +484,12 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             const int r = dual ? 128 * b + m : m;      // query row of the item
             const int t = r / G, g = r % G;
             const bool row_valid = t < it.ntok;
-            // ---- stage Q with the 128-byte swizzle the MMA descriptor expects
+            // ---- stage Q with the 128-byte swizzle the MMA descriptor expects (the previous item's
+            // epilogue used the Q tiles as its output staging area: wait until every warp is through)
+            if (item_no > 0) {
+                ok = mbar_wait_warp(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 36);
+                if (!ok) break;
+            }
             if (dual) {
 #pragma unroll
                 for (int c = 0; c < 16; ++c)
@@ -501,21 +502,23 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             }
             fence_async_smem();
             mbar_arrive(bar(kQFull));
-            it_next = load_titem(p, ii + 1, i1);
+            it_next = load_titem(p.works + ii + 1, ii + 1 < i1);
             const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
             float m_ref = -INFINITY;                     // reference maximum (log2 domain)
             float2 l2 = make_float2(0.f, 0.f);           // running sum of P, two partial sums
-            int mine = 0;                                // steps of this group so far in this item
-            for (int j = dual ? 0 : b; j < ntiles && ok; j += dual ? 1 : 2) {
+            int mine = 0;                                // tiles of this group so far in this item
+            for (int j = dual ? 0 : b; j < ntiles && ok; j += dual ? 1 : 2, ++mine) {
                 const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                for (int h = 0; h * 4 < npg && ok; ++h, ++mine) {
-                    const int u = cnt + mine, buf = u & 1;
+                // S[b] complete; it was issued after the P V of this group's previous tile finished, so
+                // O[b] is at rest as well
+                ok = mbar_wait_warp(bar(kSFull0 + 2 * b), (uint32_t)(cnt + mine) & 1u, abort_flag, p.status, 31);
+                if (!ok) break;
+                tc_fence_after();
+                // the tile is handled in two halves of 64 keys (register budget)
+                for (int h = 0; h * 4 < npg; ++h) {
                     const int base = it.kv0 + j * kTile + h * kSub;
                     const int vis = max(0, min(kSub, lim_row - base));      // visible columns of this row
-                    const uint32_t sb = s_addr + 64u * (uint32_t)buf;
-                    ok = mbar_wait_warp(bar(kSFull0 + 2 * b + buf), (uint32_t)(u >> 1) & 1u, abort_flag, p.status, 31);
-                    if (!ok) break;
-                    tc_fence_after();
+                    const uint32_t sb = s_addr + 64u * (uint32_t)h;
                     uint32_t rr[64];
                     tmem_ld32(sb, *reinterpret_cast<uint32_t(*)[32]>(&rr[0]));
                     tmem_ld32(sb + 32u, *reinterpret_cast<uint32_t(*)[32]>(&rr[32]));
@@ -541,8 +544,8 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     cmax = fmaxf(cmax, xv(63));
                     // x is relative to m_ref (to 0 while the row has no reference yet: then any visible key sets it)
                     if (__any_sync(0xffffffffu, cmax > (m_ref == -INFINITY ? -INFINITY : kRescaleThreshold))) {
-                        // Move the reference maximum (rare after the first step): rescale the running sum
-                        // and, once the P V of the previous step has landed, O[b]; shift this step's x.
+                        // Move the reference maximum (rare after the first tile): rescale the running sum, the
+                        // half of P already written for this tile and O[b], and shift this half's x.
                         const float m_new = cmax == -INFINITY ? m_ref : fmaxf(m_ref, m_use + cmax);
                         const float scale = m_new == -INFINITY ? 1.f : fast_exp2(m_ref - m_new);
                         const float shift = (m_new == -INFINITY ? 0.f : m_new) - m_use;
@@ -552,10 +555,20 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                         const float2 ns2 = make_float2(-shift, -shift);
 #pragma unroll
                         for (int e = 0; e < 32; ++e) x[e] = __fadd2_rn(x[e], ns2);
+                        tmem_wait_st();
+                        if (h > 0) {
+#pragma unroll 1
+                            for (int cc = 0; cc < 2; ++cc) {
+                                uint32_t pk[16];
+                                tmem_ld16(s_addr + 16u * cc, pk);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int e = 0; e < 16; ++e)
+                                    pk[e] = pack_bf16x2(bf16_lo(pk[e]) * scale, bf16_hi(pk[e]) * scale);
+                                tmem_st16(s_addr + 16u * cc, pk);
+                            }
+                        }
                         if (mine > 0) {
-                            ok = mbar_wait_warp(bar(kPvDone0 + 2 * b + (buf ^ 1)), (uint32_t)((u - 1) >> 1) & 1u, abort_flag, p.status, 32);
-                            if (!ok) break;
-                            tc_fence_after();
 #pragma unroll 1
                             for (int cc = 0; cc < 8; ++cc) {
                                 uint32_t ro[16];
@@ -565,10 +578,11 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                                 for (int e = 0; e < 16; ++e) ro[e] = __float_as_uint(__uint_as_float(ro[e]) * scale);
                                 tmem_st16(o_addr + 16u * cc, ro);
                             }
-                            tmem_wait_st();
                         }
+                        tmem_wait_st();
                     }
-                    // P = exp2(x) as packed bf16 over the first 32 columns of the buffer
+                    // P = exp2(x) as packed bf16: half h of the tile goes to columns [32 h, 32 h + 32) of
+                    // the buffer, which this thread has already read
                     uint32_t pk[32];
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
@@ -576,21 +590,20 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                         l2 = __fadd2_rn(l2, pe);
                         pk[e] = pack_bf16x2(pe.x, pe.y);
                     }
-                    tmem_st16(sb, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
-                    tmem_st16(sb + 16u, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
-                    tmem_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(bar(kPFull0 + 2 * b + buf));
+                    tmem_st16(s_addr + 32u * (uint32_t)h, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
+                    tmem_st16(s_addr + 32u * (uint32_t)h + 16u, *reinterpret_cast<uint32_t(*)[16]>(&pk[16]));
                 }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(kPFull0 + 2 * b));
             }
             if (!ok) break;
             const float l_sum = l2.x + l2.y;
             load_q(it_next, q_next);        // in flight during the epilogue
-            // ---- epilogue.  The groups' (max, sum) go through columns 0-1 of their first S buffer; the S
-            // buffers are idle from the group's last P V until the next item's first Q K^T.
+            // ---- epilogue.  The groups' (max, sum) go through columns 0-1 of their S buffers, which are
+            // idle from the group's last P V until the next item's first Q K^T.
             if (mine > 0) {
-                const int ul = cnt + mine - 1;
-                ok = mbar_wait_warp(bar(kPvDone0 + 2 * b + (ul & 1)), (uint32_t)(ul >> 1) & 1u, abort_flag, p.status, 34);
+                ok = mbar_wait_warp(bar(kPvDone0 + 2 * b), (uint32_t)(cnt + mine - 1) & 1u, abort_flag, p.status, 34);
                 if (!ok) break;
                 tc_fence_after();
             }
@@ -630,6 +643,29 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 c_begin = 2 * b; c_end = 2 * b + 2;
             }
             const bool use0 = __any_sync(0xffffffffu, w0 != 0.f), use1 = __any_sync(0xffffffffu, w1 != 0.f);
+            // A thread holds one row, but a row-per-thread store touches 32 lines per instruction: the
+            // warp passes each 128-byte slice of its 32 rows through shared memory (its own rows of the Q
+            // tile, which no MMA reads any more; 16-byte pieces XOR-swizzled by row) and writes whole lines.
+            const int w4 = warp & 3;
+            uint8_t* stage = smem + kOffQ + (dual ? b * kTileBytes : b * kHalfBytes) + w4 * 32 * 128;
+            const int row_base = (dual ? 128 * b : 0) + 32 * w4;      // item row of the warp's first thread
+            const bool final_out = it.partial_row0 < 0;
+            auto flush = [&](int byte0) {      // byte0: offset of the slice inside an output row
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int row = 4 * i + (lane >> 3), pc = lane & 7;
+                    const uint4 v = *reinterpret_cast<const uint4*>(stage + row * 128 + ((pc ^ (row & 7)) << 4));
+                    const int ri = row_base + row, tt = ri / G, gg = ri % G;
+                    if (tt < it.ntok) {
+                        uint8_t* dst = final_out
+                            ? reinterpret_cast<uint8_t*>(out + ((size_t)(it.q_row0 + tt) * Hq + (size_t)it.kv_head * G + gg) * kD)
+                            : reinterpret_cast<uint8_t*>(p.partial_o + (((size_t)it.partial_row0 + tt) * G + gg) * kD);
+                        *reinterpret_cast<uint4*>(dst + byte0 + pc * 16) = v;
+                    }
+                }
+                __syncwarp();
+            };
 #pragma unroll 1
             for (int c = c_begin; c < c_end; ++c) {
                 float acc[32];
@@ -653,19 +689,22 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                         for (int e = 0; e < 32; ++e) acc[e] = fmaf(__uint_as_float(ro[e]), w1, acc[e]);
                     }
                 }
-                if (row_valid) {
-                    if (it.partial_row0 < 0) {
-                        uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)(it.q_row0 + t) * Hq + hq) * kD + c * 32);
+                uint8_t* mine_row = stage + lane * 128;
+                if (final_out) {
+                    // 32 columns -> 64 bytes of bf16: pieces 4 (c & 1) .. + 3 of a 64-column slice
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            dst[k] = make_uint4(pack_bf16x2(acc[8 * k], acc[8 * k + 1]), pack_bf16x2(acc[8 * k + 2], acc[8 * k + 3]),
-                                                pack_bf16x2(acc[8 * k + 4], acc[8 * k + 5]), pack_bf16x2(acc[8 * k + 6], acc[8 * k + 7]));
-                    } else {
-                        float4* dst = reinterpret_cast<float4*>(p.partial_o + (prow * G + g) * kD + c * 32);
+                    for (int k = 0; k < 4; ++k)
+                        *reinterpret_cast<uint4*>(mine_row + ((((c & 1) * 4 + k) ^ (lane & 7)) << 4)) =
+                            make_uint4(pack_bf16x2(acc[8 * k], acc[8 * k + 1]), pack_bf16x2(acc[8 * k + 2], acc[8 * k + 3]),
+                                       pack_bf16x2(acc[8 * k + 4], acc[8 * k + 5]), pack_bf16x2(acc[8 * k + 6], acc[8 * k + 7]));
+                    if (c & 1) flush((c >> 1) * 128);
+                } else {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            dst[k] = make_float4(acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]);
-                    }
+                    for (int k = 0; k < 8; ++k)
+                        *reinterpret_cast<uint4*>(mine_row + ((k ^ (lane & 7)) << 4)) =
+                            make_uint4(__float_as_uint(acc[4 * k]), __float_as_uint(acc[4 * k + 1]),
+                                       __float_as_uint(acc[4 * k + 2]), __float_as_uint(acc[4 * k + 3]));
+                    flush(c * 128);
                 }
             }
             if (row_valid && (dual || b == 0)) {

@@ -209,17 +209,22 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
 
     if (warp >= kWarps) {
         if constexpr (!FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
+        else asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsProducer));      // idled with 24 so far
         if (warp > kWarps) return;      // the other warps of the producer's warpgroup have nothing to do
         // ------------------------------------------------------------------ producer warp
         // The page ids of the next 32 pages (8 tiles) and the descriptors of the next two items are
         // fetched ahead of use, so that no global-load latency sits between two tiles.
         struct PItem { int kv0, kv_end, q_row0, kv_head, partial_row, page0; };
         int n = 0;
-        const int i0 = p.cta_indptr_cuda[blockIdx.x], i1 = p.cta_indptr_cuda[blockIdx.x + 1];
+        // the CTA's header gives its item range, its first item and that item's first 32 page ids in
+        // one round trip to memory
+        const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
+        const int i0 = head[2], i1 = head[3];
         auto load_item = [&](int ii) {
             PItem r{0, 0, 0, 0, -1, 0};
             if (ii < i1) {
-                const int4* src = reinterpret_cast<const int4*>(p.works + ii);
+                const int4* src = ii == i0 ? reinterpret_cast<const int4*>(head + kHeadWorkCuda)
+                                           : reinterpret_cast<const int4*>(p.works + ii);
                 const int4 a = __ldg(src), b = __ldg(src + 1);
                 r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z;
                 r.kv_head = b.y; r.partial_row = b.z; r.page0 = b.w;
@@ -235,7 +240,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         constexpr int kGroupTiles = 32 / kPagesPerTile;
         bool ok = true;
         PItem cur = load_item(i0), nxt = load_item(i0 + 1);
-        int pages_cur = cur.kv_end > 0 ? load_pages(cur, 0) : 0;
+        int pages_cur = head[kHeadPagesCuda + lane];
         for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
             const PItem after = load_item(ii + 2);
             const int ntiles = (cur.kv_end - cur.kv0 + kTileTok - 1) / kTileTok;

@@ -50,6 +50,13 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = aligned_smem(smem_raw);
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
+    const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
+    if (head[0] == head[1]) {
+        // no span tiles for this CTA: straight to its decode rows, without the tensor-memory set-up
+        pdl_wait();
+        dec::decode_body<tc::kD, G, false>(p, &kv_map, q, out, lse, S, smem);
+        return;
+    }
     tc::tc_body<G, true>(p, q, pool, out, lse, smem);
     __syncthreads();      // tensor memory released, shared memory free for the second phase
     dec::decode_body<tc::kD, G, true>(p, &kv_map, q, out, lse, S, smem);

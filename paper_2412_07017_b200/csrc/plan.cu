@@ -49,7 +49,7 @@ static int default_tensor_min_rows() { return 32; }
 // Sizes of the sections of the packed blob (identical offsets on host and device).
 struct BlobLayout {
     size_t off_q_indptr, off_kv_len, off_page_indptr, off_page_indices, off_row_seq, off_units,
-        off_items, off_works, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
+        off_items, off_works, off_heads, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
 };
 
 static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64_t n_units,
@@ -67,6 +67,7 @@ static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64
     L.off_units = take(sizeof(Unit) * (size_t)std::max<int64_t>(n_units, 1));
     L.off_items = take(sizeof(Item) * (size_t)std::max<int64_t>(n_items, 1));
     L.off_works = take(sizeof(Work) * (size_t)std::max<int64_t>(n_items, 1));
+    L.off_heads = take(sizeof(int32_t) * kHeadWords * (size_t)std::max(ctas_cuda, ctas_tensor));
     L.off_cta_cuda = take(sizeof(int32_t) * (size_t)(ctas_cuda + 1));
     L.off_cta_tensor = take(sizeof(int32_t) * (size_t)(ctas_tensor + 1));
     L.off_split = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_split, 1));
@@ -216,9 +217,9 @@ struct PathCost {
     int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
 };
 // (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
-constexpr PathCost kTensorCost{128, 1500, 4000, 3000};
-constexpr PathCost kCudaCost{96, 1260, 1100, 6000};
-constexpr int64_t kTensorDualTileNs = 1900;   // a KV tile of an item with two row tiles (more than 128 rows)
+constexpr PathCost kTensorCost{128, 1470, 7100, 7000};
+constexpr PathCost kCudaCost{96, 1150, 1000, 5000};
+constexpr int64_t kTensorDualTileNs = 3170;   // a KV tile of an item with two row tiles (more than 128 rows)
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
 // then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
@@ -231,25 +232,26 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
                   std::vector<int32_t>& item_cta) {
     struct Piece { Item it; int32_t cta; };
     std::vector<Piece> best[2];
-    int64_t best_max = -1;
     const std::vector<int>* ids[2] = {&ids_tensor, &ids_cuda};
     const PathCost cost[2] = {kTensorCost, kCudaCost};
     auto tile_ns = [&](int path, int id) {
         return path == 0 && units[id].u.ntok * group > 128 ? kTensorDualTileNs : cost[path].tile_ns;
     };
+    // Lower bound of the makespan: all work, one start per unit, one phase start per CTA.
     int64_t total = 0;
     for (int path = 0; path < 2; ++path)
         for (int id : *ids[path])
             total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * tile_ns(path, id);
-    total += (int64_t)n_ctas * (kTensorCost.item_ns + kCudaCost.phase_ns) / 2;
-    int64_t quota = std::max<int64_t>(1, (total + n_ctas - 1) / n_ctas);
-    for (int round = 0; round < 8; ++round) {
-        std::vector<Piece> out[2];
-        std::vector<int64_t> load((size_t)n_ctas, 0);
+    // Fill the CTAs one after the other up to a load limit `cap`; returns false if the work does not
+    // fit (the last CTA would have to exceed the limit).  A unit is cut only where a CTA is full.
+    auto fill = [&](int64_t cap, std::vector<Piece> (&out)[2]) {
+        out[0].clear();
+        out[1].clear();
         int cta = 0;
-        int64_t cum = 0;      // cost laid down so far; CTA k ends where the line reaches (k + 1) * quota
+        int64_t load = 0;
         bool has_phase[2] = {false, false};
-        auto next_cta = [&]() { ++cta; has_phase[0] = has_phase[1] = false; };
+        bool fits = true;
+        auto next_cta = [&]() { ++cta; load = 0; has_phase[0] = has_phase[1] = false; };
         for (int path = 0; path < 2; ++path) {
             PathCost pc = cost[path];
             for (int id : *ids[path]) {
@@ -260,41 +262,45 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
                 while (left > 0) {
                     const bool last_cta = cta + 1 >= n_ctas;
                     const int64_t start = pc.item_ns + (has_phase[path] ? 0 : pc.phase_ns);
-                    const int64_t room = (int64_t)(cta + 1) * quota - cum - start;
+                    const int64_t room = cap - load - start;
                     int64_t take;
-                    if (last_cta || left * pc.tile_ns <= room + pc.item_ns) {
-                        take = left;                       // finishing here is cheaper than a new item elsewhere
-                    } else if (room < pc.tile_ns / 2 && load[(size_t)cta] > 0) {
-                        next_cta();
+                    if (last_cta) {
+                        take = left;
+                        if (load + start + take * pc.tile_ns > cap) fits = false;
+                    } else if (left * pc.tile_ns <= room + pc.item_ns / 2) {
+                        take = left;                     // finishing here is cheaper than another item elsewhere
+                    } else if (room < pc.tile_ns * 2 && load > 0) {
+                        next_cta();                      // not worth starting an item for so little
                         continue;
                     } else {
-                        take = std::max<int64_t>(1, (room + pc.tile_ns / 2) / pc.tile_ns);   // nearest: errors average out
+                        take = std::max<int64_t>(1, room / pc.tile_ns);
                     }
                     const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
                     out[path].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
-                    load[(size_t)cta] += start + take * pc.tile_ns;
-                    cum += start + take * pc.tile_ns;
+                    load += start + take * pc.tile_ns;
                     has_phase[path] = true;
                     left -= take;
                     k0 = k1;
                     ++c;
-                    while (cta + 1 < n_ctas && cum >= (int64_t)(cta + 1) * quota) next_cta();
+                    if (!last_cta && left > 0) next_cta();
                 }
             }
         }
-        int64_t mx = 0, sum = 0;
-        for (int64_t l : load) { mx = std::max(mx, l); sum += l; }
-        if (best_max < 0 || mx < best_max) {
-            best_max = mx;
-            best[0] = out[0];
-            best[1] = out[1];
+        return fits;
+    };
+    // Smallest limit that fits, by bisection (the loads are monotone in the limit up to rounding).
+    int64_t lo = std::max<int64_t>(1, total / n_ctas), hi = 2 * lo + kTensorCost.item_ns + kTensorCost.phase_ns + kCudaCost.phase_ns;
+    while (!fill(hi, best)) hi *= 2;
+    for (int iter = 0; iter < 24 && hi - lo > 50; ++iter) {
+        const int64_t mid = (lo + hi) / 2;
+        std::vector<Piece> trial[2];
+        if (fill(mid, trial)) {
+            hi = mid;
+            best[0].swap(trial[0]);
+            best[1].swap(trial[1]);
+        } else {
+            lo = mid;
         }
-        // next round: aim at the mean of what this round really cost; if the last CTA, which takes
-        // whatever is left, still ends up above the others, spread its excess over all of them
-        const int64_t mean = (sum + n_ctas - 1) / n_ctas;
-        const int64_t over = load[(size_t)n_ctas - 1] - quota;
-        quota = round == 0 ? mean : quota + (over > 0 ? (over + n_ctas - 1) / n_ctas : 0);
-        if (round > 0 && over <= 0) break;
     }
     // emit: CUDA-core items first, then tensor items; chunk counts per unit
     cta_indptr_cuda.assign((size_t)n_ctas + 1, 0);
@@ -494,6 +500,8 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     Unit* h_units = (Unit*)(hb + L.off_units);
     for (size_t i = 0; i < units.size(); ++i) h_units[i] = units[i].u;
     if (n_items > 0) std::memcpy(hb + L.off_items, items.data(), sizeof(Item) * (size_t)n_items);
+    int32_t* h_heads = (int32_t*)(hb + L.off_heads);
+    std::memset(h_heads, 0, sizeof(int32_t) * kHeadWords * (size_t)std::max(ctas_cuda, ctas_tensor));
     Work* h_works = (Work*)(hb + L.off_works);
     for (int i = 0; i < n_items; ++i) {
         const Item& it = items[(size_t)i];
@@ -508,6 +516,23 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
         w.partial_row0 = u.partial_base < 0 ? -1 : u.partial_base + it.chunk * u.ntok;
         w.page0 = u.page_base + it.kv0 / kPage;
         h_works[i] = w;
+    }
+    for (int c = 0; c < std::max(ctas_cuda, ctas_tensor); ++c) {
+        int32_t* h = h_heads + (size_t)c * kHeadWords;
+        const int32_t range[4] = {c < ctas_tensor ? cta_indptr_tensor[(size_t)c] : 0,
+                                  c < ctas_tensor ? cta_indptr_tensor[(size_t)c + 1] : 0,
+                                  c < ctas_cuda ? cta_indptr_cuda[(size_t)c] : 0,
+                                  c < ctas_cuda ? cta_indptr_cuda[(size_t)c + 1] : 0};
+        std::memcpy(h, range, sizeof(range));
+        for (int path = 0; path < 2; ++path) {
+            const int first = range[2 * path], last = range[2 * path + 1];
+            if (first >= last) continue;
+            const Work& w = h_works[first];
+            std::memcpy(h + (path == 0 ? kHeadWorkTensor : kHeadWorkCuda), &w, sizeof(Work));
+            const int npg = (w.kv_end - w.kv0 + kPage - 1) / kPage;
+            for (int k = 0; k < 32 && k < npg; ++k)
+                h[(path == 0 ? kHeadPagesTensor : kHeadPagesCuda) + k] = batch->page_indices[w.page0 + k];
+        }
     }
     std::memcpy(hb + L.off_cta_cuda, cta_indptr_cuda.data(), sizeof(int32_t) * (size_t)(ctas_cuda + 1));
     std::memcpy(hb + L.off_cta_tensor, cta_indptr_tensor.data(),
@@ -542,6 +567,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     d.units = (const Unit*)dp(L.off_units);
     d.items = (const Item*)dp(L.off_items);
     d.works = (const Work*)dp(L.off_works);
+    d.cta_heads = (const int32_t*)dp(L.off_heads);
     d.cta_indptr_cuda = (const int32_t*)dp(L.off_cta_cuda);
     d.cta_indptr_tensor = (const int32_t*)dp(L.off_cta_tensor);
     d.split_units = (const int32_t*)dp(L.off_split);

@@ -44,6 +44,14 @@ struct alignas(16) Work {
     int32_t page0;         // index into page_indices of the page that holds key kv0
 };
 
+// Per persistent CTA, one 384-byte header that holds everything the CTA needs to issue its first
+// loads after a single round trip to memory: words 0-3 its item ranges (tensor first, last;
+// CUDA-core first, last), words 8-15 the Work record of its first tensor item, words 16-23 that of
+// its first CUDA-core item, words 32-63 the first 32 page ids of the first tensor item and words
+// 64-95 those of the first CUDA-core item.
+constexpr int kHeadWords = 96;
+constexpr int kHeadWorkTensor = 8, kHeadWorkCuda = 16, kHeadPagesTensor = 32, kHeadPagesCuda = 64;
+
 // Pointers into the device workspace, passed to kernels by value.
 struct DevPlan {
     const int32_t* q_indptr;
@@ -54,6 +62,7 @@ struct DevPlan {
     const Unit* units;
     const Item* items;               // CUDA-core items first (grouped by CTA), then tensor items
     const Work* works;               // [num_items] the same items, resolved for the kernels
+    const int32_t* cta_heads;        // [num_ctas][kHeadWords], see above
     const int32_t* cta_indptr_cuda;  // [num_ctas_cuda + 1] into items
     const int32_t* cta_indptr_tensor;// [num_ctas_tensor + 1] into items (absolute indices)
     const int32_t* split_units;      // [num_split_units] unit ids that need a merge
