@@ -24,12 +24,12 @@ kv_append_kernel(DevPlan p, const uint4* __restrict__ k_new, const uint4* __rest
         rest /= p.num_kv_heads;
         const int which = (int)(rest & 1);
         const int r = (int)(rest >> 1);
-        const int b = p.row_seq[r];
-        const int pos = p.kv_len_before[b] + (r - p.q_indptr[b]);
-        const int64_t page = p.page_indices[p.page_indptr[b] + pos / kPage];
-        const uint4* src = (which ? v_new : k_new) + ((size_t)r * p.num_kv_heads + h) * vpr + vec;
-        const size_t dst = pool_row_offset(page, which, h, pos % kPage, p.num_kv_heads, p.head_dim) / 8 + vec;
-        pool[dst] = *src;
+        // the planner resolved the row's page and slot (position ctx_b + i through the page table), so
+        // the slot and the source row are fetched side by side instead of through four dependent loads
+        const int64_t ps = __ldg(p.row_slot + r);
+        const uint4 val = ldg_nc_v4((which ? v_new : k_new) + ((size_t)r * p.num_kv_heads + h) * vpr + vec);
+        const size_t dst = pool_row_offset(ps / kPage, which, h, (int)(ps % kPage), p.num_kv_heads, p.head_dim) / 8 + vec;
+        pool[dst] = val;
     }
 }
 

@@ -48,7 +48,7 @@ static int default_tensor_min_rows() { return 32; }
 
 // Sizes of the sections of the packed blob (identical offsets on host and device).
 struct BlobLayout {
-    size_t off_q_indptr, off_kv_len, off_page_indptr, off_page_indices, off_row_seq, off_units,
+    size_t off_q_indptr, off_kv_len, off_page_indptr, off_page_indices, off_row_seq, off_row_slot, off_units,
         off_items, off_works, off_heads, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
 };
 
@@ -64,6 +64,7 @@ static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64
     L.off_page_indptr = take(sizeof(int32_t) * (size_t)(batch + 1));
     L.off_page_indices = take(sizeof(int32_t) * (size_t)std::max<int64_t>(total_pages, 1));
     L.off_row_seq = take(sizeof(int32_t) * (size_t)std::max(total_q, 1));
+    L.off_row_slot = take(sizeof(int64_t) * (size_t)std::max(total_q, 1));
     L.off_units = take(sizeof(Unit) * (size_t)std::max<int64_t>(n_units, 1));
     L.off_items = take(sizeof(Item) * (size_t)std::max<int64_t>(n_items, 1));
     L.off_works = take(sizeof(Work) * (size_t)std::max<int64_t>(n_items, 1));
@@ -457,7 +458,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     const int n_items = (int)items.size();
 
     // ---- partial rows ------------------------------------------------------------------------
-    std::vector<int32_t> split_units, merge_blocks;   // merge block: 4 (token, head) rows of a split unit
+    std::vector<int32_t> split_units, merge_blocks;   // merge block: 32 (token, head) rows of a split unit
     int64_t partial_rows = 0;
     for (size_t i = 0; i < units.size(); ++i) {
         if (units[i].u.n_chunks > 1) {
@@ -465,7 +466,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
             partial_rows += (int64_t)units[i].u.n_chunks * units[i].u.ntok;
             split_units.push_back((int32_t)i);
             if (i >= (size_t)(INT32_MAX >> 6)) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
-            for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
+            for (int rb = 0; rb * 32 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
             if (partial_rows > INT32_MAX / 2) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
         }
     }
@@ -495,8 +496,13 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     if (total_pages > 0)
         std::memcpy(hb + L.off_page_indices, batch->page_indices, sizeof(int32_t) * (size_t)total_pages);
     int32_t* row_seq = (int32_t*)(hb + L.off_row_seq);
+    int64_t* row_slot = (int64_t*)(hb + L.off_row_slot);
     for (int b = 0; b < B; ++b)
-        for (int r = q_indptr[b]; r < q_indptr[b + 1]; ++r) row_seq[r] = b;
+        for (int r = q_indptr[b]; r < q_indptr[b + 1]; ++r) {
+            row_seq[r] = b;
+            const int pos = batch->kv_len_before[b] + (r - q_indptr[b]);
+            row_slot[r] = (int64_t)batch->page_indices[page_indptr[b] + pos / P] * P + pos % P;
+        }
     Unit* h_units = (Unit*)(hb + L.off_units);
     for (size_t i = 0; i < units.size(); ++i) h_units[i] = units[i].u;
     if (n_items > 0) std::memcpy(hb + L.off_items, items.data(), sizeof(Item) * (size_t)n_items);
@@ -564,6 +570,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     d.page_indptr = (const int32_t*)dp(L.off_page_indptr);
     d.page_indices = (const int32_t*)dp(L.off_page_indices);
     d.row_seq = (const int32_t*)dp(L.off_row_seq);
+    d.row_slot = (const int64_t*)dp(L.off_row_slot);
     d.units = (const Unit*)dp(L.off_units);
     d.items = (const Item*)dp(L.off_items);
     d.works = (const Work*)dp(L.off_works);
