@@ -1,6 +1,6 @@
 // Split-KV merge: combine the per-chunk (normalised output, log-sum-exp) pairs of one row,
 //     LSE = log sum_c exp(LSE_c),   O = sum_c exp(LSE_c - LSE) O_c.
-// One warp per (token, head) row that was split, 32 rows per CTA (the planner lists the row
+// One warp per (token, head) row that was split, 4 rows per CTA (the planner lists the row
 // blocks); chunks are added in chunk order, so the result does not depend on which CTA produced
 // which chunk or on scheduling.
 #include "common.cuh"
@@ -8,10 +8,11 @@
 
 namespace asynclm {
 
-// A block takes 32 (token, head) rows of one split unit, two per warp: few fat blocks, so that the
-// whole grid is resident at once and block dispatch does not dominate this microsecond-sized kernel.
-constexpr int kMergeThreads = 512;
-constexpr int kMergeRows = 32;
+// A block takes 4 (token, head) rows of one split unit, one per warp.  (Measured: blocks of 512
+// threads with two rows per warp were slower; late blocks of a dependent grid are dispatched slowly,
+// so small blocks that fit beside each other early do better.)
+constexpr int kMergeThreads = 128;
+constexpr int kMergeRows = 4;
 
 template <int D>
 __global__ void __launch_bounds__(kMergeThreads)
@@ -22,10 +23,19 @@ lse_merge_kernel(DevPlan p, __nv_bfloat16* __restrict__ out, float* __restrict__
     // the plan was uploaded before the attention kernel started: read it while that kernel drains
     const int entry = p.merge_blocks[blockIdx.x];
     const Unit u = p.units[entry >> 6];
+    const int pair = (entry & 63) * kMergeRows + (threadIdx.x >> 5);
+    if (pair < u.ntok * G) {
+        // Touch the row's partial results ahead of the wait: the data is not final yet, but the address
+        // translations are, and a first touch from this SM costs more than the L2 hit that follows.
+        const size_t prow = (size_t)u.partial_base + pair / G;
+        for (int c = lane; c < u.n_chunks; c += 32) {
+            const size_t r = (prow + (size_t)c * u.ntok) * G + pair % G;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.partial_lse + r));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.partial_o + r * D));
+        }
+    }
     pdl_wait();     // the partial results are complete and visible from here on
-#pragma unroll 1
-  for (int half = 0; half < 2; ++half) {
-    const int pair = (entry & 63) * kMergeRows + (threadIdx.x >> 5) + 16 * half;
+  {
     if (pair >= u.ntok * G) return;
     const int t = pair / G, g = pair % G;
     const int n = u.n_chunks;

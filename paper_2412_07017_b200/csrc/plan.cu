@@ -218,9 +218,9 @@ struct PathCost {
     int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
 };
 // (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
-constexpr PathCost kTensorCost{128, 1470, 7100, 7000};
-constexpr PathCost kCudaCost{96, 1150, 1000, 5000};
-constexpr int64_t kTensorDualTileNs = 3170;   // a KV tile of an item with two row tiles (more than 128 rows)
+constexpr PathCost kTensorCost{128, 1530, 6200, 5700};
+constexpr PathCost kCudaCost{96, 1290, 900, 4100};
+constexpr int64_t kTensorDualTileNs = 3130;   // a KV tile of an item with two row tiles (more than 128 rows)
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
 // then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
@@ -243,43 +243,84 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     for (int path = 0; path < 2; ++path)
         for (int id : *ids[path])
             total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * tile_ns(path, id);
-    // Fill the CTAs one after the other up to a load limit `cap`; returns false if the work does not
-    // fit (the last CTA would have to exceed the limit).  A unit is cut only where a CTA is full.
+    // Deal the work under a per-CTA load limit `cap`; returns false if it does not fit.
+    //   Span units first, whole wherever possible (an unsplit unit writes final bf16 rows: no fp32
+    // partial rows, no merge): largest first, each into the fullest span CTA that still has room for
+    // it, else into a fresh CTA; a unit larger than a CTA's share is cut into equal pieces.
+    //   Decode units then fill every CTA up to the limit in CTA order; a unit is cut only where a
+    // CTA is full.
+    std::vector<int> tensor_order(ids_tensor);
+    auto unit_tiles = [&](int path, int id) { return (units[id].n_keys + cost[path].gran - 1) / cost[path].gran; };
+    std::stable_sort(tensor_order.begin(), tensor_order.end(), [&](int x, int y) {
+        return unit_tiles(0, x) * tile_ns(0, x) > unit_tiles(0, y) * tile_ns(0, y);
+    });
     auto fill = [&](int64_t cap, std::vector<Piece> (&out)[2]) {
         out[0].clear();
         out[1].clear();
-        int cta = 0;
-        int64_t load = 0;
-        bool has_phase[2] = {false, false};
         bool fits = true;
-        auto next_cta = [&]() { ++cta; load = 0; has_phase[0] = has_phase[1] = false; };
-        for (int path = 0; path < 2; ++path) {
-            PathCost pc = cost[path];
-            for (int id : *ids[path]) {
-                pc.tile_ns = tile_ns(path, id);
-                int64_t left = (units[id].n_keys + pc.gran - 1) / pc.gran;   // tiles left
+        std::vector<int64_t> load((size_t)n_ctas, 0);
+        int used = 0;                                   // CTAs that hold span work: [0, used)
+        {
+            const PathCost& pc = cost[0];
+            for (int id : tensor_order) {
+                const int64_t tns = tile_ns(0, id);
+                const int64_t tiles = unit_tiles(0, id);
+                const int64_t fresh_room = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / tns);   // tiles a fresh CTA takes
+                const int64_t pieces = (tiles + fresh_room - 1) / fresh_room;
+                int64_t k0 = 0;
+                for (int64_t c = 0; c < pieces; ++c) {
+                    const int64_t take = tiles / pieces + (c < tiles % pieces ? 1 : 0);
+                    const int64_t need = pc.item_ns + take * tns;
+                    int best_cta = -1;
+                    for (int k = 0; k < used; ++k)
+                        if (load[(size_t)k] + need <= cap && (best_cta < 0 || load[(size_t)k] > load[(size_t)best_cta])) best_cta = k;
+                    if (best_cta < 0) {
+                        if (used < n_ctas) {
+                            best_cta = used++;
+                            load[(size_t)best_cta] = pc.phase_ns;
+                        } else {
+                            fits = false;
+                            best_cta = 0;
+                            for (int k = 1; k < n_ctas; ++k) if (load[(size_t)k] < load[(size_t)best_cta]) best_cta = k;
+                        }
+                    }
+                    const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
+                    out[0].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c}, (int32_t)best_cta});
+                    load[(size_t)best_cta] += need;
+                    k0 = k1;
+                }
+            }
+            std::stable_sort(out[0].begin(), out[0].end(), [](const Piece& x, const Piece& y) { return x.cta < y.cta; });
+        }
+        {
+            PathCost pc = cost[1];
+            int cta = 0;
+            bool has_phase = false;
+            auto next_cta = [&]() { ++cta; has_phase = false; };
+            for (int id : *ids[1]) {
+                int64_t left = unit_tiles(1, id);
                 int64_t k0 = 0;
                 int c = 0;
                 while (left > 0) {
                     const bool last_cta = cta + 1 >= n_ctas;
-                    const int64_t start = pc.item_ns + (has_phase[path] ? 0 : pc.phase_ns);
-                    const int64_t room = cap - load - start;
+                    const int64_t start = pc.item_ns + (has_phase ? 0 : pc.phase_ns);
+                    const int64_t room = cap - load[(size_t)cta] - start;
                     int64_t take;
                     if (last_cta) {
                         take = left;
-                        if (load + start + take * pc.tile_ns > cap) fits = false;
+                        if (load[(size_t)cta] + start + take * pc.tile_ns > cap) fits = false;
                     } else if (left * pc.tile_ns <= room + pc.item_ns / 2) {
                         take = left;                     // finishing here is cheaper than another item elsewhere
-                    } else if (room < pc.tile_ns * 2 && load > 0) {
+                    } else if (room < pc.tile_ns * 2) {
                         next_cta();                      // not worth starting an item for so little
                         continue;
                     } else {
                         take = std::max<int64_t>(1, room / pc.tile_ns);
                     }
                     const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
-                    out[path].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
-                    load += start + take * pc.tile_ns;
-                    has_phase[path] = true;
+                    out[1].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
+                    load[(size_t)cta] += start + take * pc.tile_ns;
+                    has_phase = true;
                     left -= take;
                     k0 = k1;
                     ++c;
@@ -314,7 +355,7 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
             items.push_back(pz.it);
             item_cta.push_back(pz.cta);
             count[(size_t)pz.cta]++;
-            units[pz.it.unit].u.n_chunks = pz.it.chunk + 1;
+            units[pz.it.unit].u.n_chunks = std::max(units[pz.it.unit].u.n_chunks, pz.it.chunk + 1);
         }
         int32_t at = first;
         for (int k = 0; k < n_ctas; ++k) {
@@ -458,7 +499,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     const int n_items = (int)items.size();
 
     // ---- partial rows ------------------------------------------------------------------------
-    std::vector<int32_t> split_units, merge_blocks;   // merge block: 32 (token, head) rows of a split unit
+    std::vector<int32_t> split_units, merge_blocks;   // merge block: 4 (token, head) rows of a split unit
     int64_t partial_rows = 0;
     for (size_t i = 0; i < units.size(); ++i) {
         if (units[i].u.n_chunks > 1) {
@@ -466,7 +507,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
             partial_rows += (int64_t)units[i].u.n_chunks * units[i].u.ntok;
             split_units.push_back((int32_t)i);
             if (i >= (size_t)(INT32_MAX >> 6)) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
-            for (int rb = 0; rb * 32 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
+            for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
             if (partial_rows > INT32_MAX / 2) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
         }
     }

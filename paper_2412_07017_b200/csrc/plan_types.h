@@ -67,7 +67,7 @@ struct DevPlan {
     const int32_t* cta_indptr_cuda;  // [num_ctas_cuda + 1] into items
     const int32_t* cta_indptr_tensor;// [num_ctas_tensor + 1] into items (absolute indices)
     const int32_t* split_units;      // [num_split_units] unit ids that need a merge
-    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 6) | row block: 32 (token, head) rows each
+    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 6) | row block: 4 (token, head) rows each
     float* partial_o;                // [partial_rows][G][d]
     float* partial_lse;              // [partial_rows][G]   (log2 domain)
     int32_t* status;                 // device status word
