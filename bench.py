@@ -33,7 +33,7 @@ WORKLOAD = "config2-llama3-8b-mixed-batch"       # the configuration the metric 
 WORKLOADS = {2: WORKLOAD, 3: "config3-large-batch-gqa8", 4: "config4-long-context-split-kv"}
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on this workload
 # (profiles/attn_fused_kernel_config2.md); None whenever the kernel has changed since that capture
-TRAFFIC_BYTES_PER_LAUNCH = 343_876_352
+TRAFFIC_BYTES_PER_LAUNCH = 327_289_856
 
 
 def measured_peaks():
@@ -182,7 +182,13 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    wl = W.make_config(args.config)
+    if args.decode_only:
+        # 64 sequences of the Llama-3-8B attention shape, contexts uniform in [1024, 3072], one decode
+        # token each: the CUDA-core decode kernel alone (profiling aid, not the benchmarked workload)
+        lens = np.random.default_rng(3).integers(1024, 3073, 64).tolist()
+        wl = W.make_single_step("decode-only", W.Shape(32, 8, 128, 16), lens, [1] * 64, seed=11)
+    else:
+        wl = W.make_config(args.config)
     st = wl.steps[0]
     shape = wl.shape
     by = W.algorithmic_bytes(shape, st)
@@ -316,7 +322,7 @@ def run_gpu(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": WORKLOADS[args.config], "seed": wl.seed, "batch": st.batch, "total_q": T,
+            "workload": "decode-only-64x[1024,3072]" if args.decode_only else WORKLOADS[args.config], "seed": wl.seed, "batch": st.batch, "total_q": T,
             "kv_tokens": int(plan.info["total_kv_tokens"]), "replicas": world,
             "l2": "256 MiB buffer rewritten between timed steps (untimed)",
             "us_per_step": ms_per_step * 1e3,
@@ -329,9 +335,10 @@ def run_gpu(args):
                                                "kv_chunk_tokens", "num_ctas_cuda", "num_ctas_tensor")},
         },
         "roofline": {"bound": "hbm",
-                     "kernel": "attn_fused_kernel (+ lse_merge_kernel; timed together as asynclm_attn_mixed)",
+                     "kernel": ("attn_decode_kernel" if args.decode_only else "attn_fused_kernel") +
+                               " (+ lse_merge_kernel; timed together as asynclm_attn_mixed)",
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.config == 2 else None,
+                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.config == 2 and not args.decode_only else None,
                      "algorithmic_bytes_per_launch": attn_bytes, "avg_launch_us": attn_s * 1e6},
         "e2e": {"value": world * by["kv"] / (e2e_total / e2e_steps) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d),
@@ -360,6 +367,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
                     help="synthetic configuration; 2 is the benchmark, 3 and 4 are for reference")
+    ap.add_argument("--decode-only", action="store_true",
+                    help="time a decode-only batch instead (exercises attn_decode_kernel alone)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

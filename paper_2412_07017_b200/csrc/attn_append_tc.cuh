@@ -15,11 +15,14 @@
 //                     * items with at most 128 rows: the groups take alternate KV tiles of the one
 //                       row tile and their (max, sum, O) states are merged in the epilogue like two
 //                       KV splits.
-//                   The softmax runs in place: a thread reads its row of S 32 columns at a time and
+//                   The softmax runs in place: a thread reads its row of S 64 columns at a time and
 //                   writes P as packed bf16 pairs over the columns it has already read; P V then
 //                   takes its A operand from tensor memory.  The reference maximum only moves when
-//                   a score exceeds it by 2^8; then O, the running sum and the part of P already
-//                   written are rescaled.
+//                   a score exceeds it by 2^8; then O, the running sum and the half of P already
+//                   written are rescaled.  The exponentials bound this stage (16 per clock and SM),
+//                   so everything around them is packed two values to an instruction.
+//                   At the end of an item the rows go out through the group's (now idle) Q tile in
+//                   shared memory, so that every global store writes whole 128-byte lines.
 //   warps 8, 10     producers of K tiles and of V tiles: 16-byte cp.async copies (fully coalesced,
 //                   two 256-byte rows per warp instruction) that write the 128-byte-swizzled operand
 //                   layout and complete on the slot's mbarrier.  K and V share one ring of five

@@ -155,6 +155,45 @@ def test_replay_steps_keep_state_across_steps():
         assert_close(out, lse, ref_out, ref_lse, what=f"replay step {t}")
 
 
+@pytest.mark.parametrize("Hq,Hkv,ctx,ql", [
+    (32, 8, [700, 64, 0, 129], [64, 33, 64, 40]),       # two full row tiles per (sequence, kv head), ragged second tile
+    (32, 8, [1000], [200]),                              # a span longer than one work item: several units per head
+    (16, 2, [300, 55], [32, 17]),                        # 8 heads per kv head: 256 rows from 32 tokens
+    (4, 4, [500, 20], [256, 130]),                       # one head per kv head: the row tiles are all tokens
+    (8, 2, [48, 64, 65, 127, 128, 193], [40, 40, 40, 40, 40, 40]),   # last KV tile with 1..8 pages
+])
+def test_span_row_tile_pairs(Hq, Hkv, ctx, ql):
+    """Spans whose (token, head) rows fill one row tile, exactly two, two with a ragged end, or more
+    than one work item, across the KV-tile tail lengths the two-half softmax distinguishes."""
+    shape = W.Shape(Hq, Hkv, 128, 16)
+    wl = W.make_single_step("pairs", shape, ctx, ql, seed=300 + Hq + len(ctx), interleave_pages=True)
+    run_and_check(wl, what=f"row tile pairs {Hq}/{Hkv}")
+    run_and_check(wl, what=f"row tile pairs {Hq}/{Hkv}, fixed chunks", kv_chunk_tokens=128)
+
+
+def test_scores_that_keep_growing_move_the_reference_maximum():
+    """Keys whose scores rise steadily along the context: the lazily updated softmax reference of
+    both attention paths has to move again and again (and rescale what it has accumulated)."""
+    shape = W.Shape(8, 2, 128, 16)
+    ctx, ql = [1200, 1200, 900], [40, 1, 70]
+    wl = W.make_single_step("growing", shape, ctx, ql, seed=91)
+    st = wl.steps[0]
+    d = shape.head_dim
+    u = np.ones(d, dtype=np.float32)
+    for b in range(len(ctx)):
+        n = ctx[b] + ql[b]
+        # q . k / sqrt(d) runs from about -40 to +40 over the sequence
+        alpha = np.linspace(-40.0, 40.0, n, dtype=np.float32) * np.sqrt(d) / d
+        for pos in range(ctx[b]):
+            pg = st.page_indices[st.page_indptr[b] + pos // 16]
+            wl.kv_pool[pg, 0, :, pos % 16, :] = W.f32_to_bf16_bits(alpha[pos] * u)[None, :]
+        for i in range(ql[b]):
+            st.k_new[st.q_indptr[b] + i] = W.f32_to_bf16_bits(alpha[ctx[b] + i] * u)[None, :]
+    st.q[:] = W.f32_to_bf16_bits(u)[None, None, :]
+    run_and_check(wl, what="growing scores")
+    run_and_check(wl, what="growing scores, split", kv_chunk_tokens=256)
+
+
 def test_config2_llama_batch_full_size():
     """Full-size Llama-3-8B-shaped mixed batch, default planning (the benchmarked configuration)."""
     wl = W.make_config(2)
