@@ -29,9 +29,9 @@
 //                   32 KiB slots, filled in the order the tensor core consumes them
 //                   (K0 K1 V0 K2 V1 K3 ...): a V tile is needed one softmax later than the K tile
 //                   of the same keys, and a shared ring lets whichever is due use the free slots.
-//   warps 9, 11     one thread each issues the Q K^T MMAs and the P V MMAs (two issuers, so that
-//                   one's barrier bookkeeping hides behind the other's MMAs).  Warp 9 owns the
-//                   tensor-memory allocation.
+//   warp 9          one thread issues all MMAs, a group at a time (P V of its tile, then Q K^T of its
+//                   next tile), so that the groups' softmaxes alternate instead of colliding on the
+//                   exponential unit.  The warp owns the tensor-memory allocation.  (Warp 11 idles.)
 // All hand-offs are mbarriers with bounded waits; a wait that runs out sets the plan's status word
 // and a CTA-wide abort flag, every role falls through to the common exit, and the tensor memory is
 // released there.
@@ -312,8 +312,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             const int ntiles = (cur.kv_end - cur.kv0 + kTile - 1) / kTile;
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
-                if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
-                else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
                 const int t1 = min(t0 + kGroupTiles, ntiles);
                 for (int t = t0; t < t1 && ok; ++t, ++n) {
                     const int rows = min(kTile, cur.kv_end - (cur.kv0 + t * kTile));
@@ -340,6 +338,12 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                         }
                     }
                     cp_async_arrive(bar(kRingFull0 + s));
+                    // page ids of the next group of tiles (or of the next item), requested only after this
+                    // group's first tile is on its way: the next item's descriptor may still be in flight
+                    if (t == t0) {
+                        if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
+                        else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
+                    }
                 }
                 pages_cur = pages_nxt;
             }
@@ -351,14 +355,20 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             asm volatile("cp.async.wait_all;" ::: "memory");
         }
     } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ Q K^T issuer
-        // An MMA costs about 94 cycles however narrow it is (measured), so Q K^T is issued 128 keys wide:
-        // 8 instructions per tile and group.
+        // ------------------------------------------------------------------ MMA issuer
+        // One thread issues every MMA of the CTA, in an order that lets the two softmax groups work
+        // in turns: after the P V of a group's tile it issues the Q K^T of the same group's next tile
+        // at once (MMAs of one thread execute in issue order, so the new S may overwrite the P that the
+        // P V in front of it reads), then it turns to the other group.  While the tensor core works
+        // for one group, the other group's softmax has the exponential unit to itself.
+        // An MMA costs about 94 cycles however narrow it is (measured), so Q K^T is issued 128 keys
+        // wide: 8 instructions per tile and group.
         if (lane == 0) {
             bool ok = true;
             int gt = 0;               // KV tiles before this item (all items): ring position
-            int cnt0 = 0, cnt1 = 0;   // steps handed to each softmax group so far
+            int cnt0 = 0, cnt1 = 0;   // tiles whose P V has been issued, per group: phase of the P hand-off
             int item_no = 0;
+            const uint32_t idesc_pv = instr_desc(128, 1);
             TItem it_next = load_titem(head_work, i0 < i1);
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
@@ -366,34 +376,62 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
                 const bool dual = it.ntok * G > kTile;
                 ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
-                // the S buffers hold the previous item's softmax statistics until its epilogue is over
+                // S and O of the previous item are in use until its epilogue is over
                 if (ok && item_no > 0) ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 27);
                 if (ok) tc_fence_after();
-                int local0 = 0, local1 = 0;      // tiles of this item issued to each group
-                for (int j = 0; j < ntiles && ok; ++j) {
+                auto tile_pages = [&](int j) { return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage; };
+                // S[b] <- Q[qt] K_j^T; release_k: this is the last use of the K tile
+                auto issue_qk = [&](int j, int b, bool release_k) {
                     const int pos = ring_pos_k(gt + j), s = pos % kRing;
                     ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
-                    const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                    const uint32_t idesc = instr_desc(16u * (uint32_t)npg, 0);
-                    for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
-                        const int u = b ? cnt1 : cnt0;
-                        // S[b] (and P[b] on top of it) is free once the P V of the group's previous tile is done
-                        if ((b ? local1 : local0) >= 1)
-                            ok = mbar_wait(bar(kPvDone0 + 2 * b), (uint32_t)(u - 1) & 1u, abort_flag, p.status, 23);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
-                        const uint32_t qbase = sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u);
-                        const uint32_t kbase = sbase + kOffRing + s * kTileBytes;
+                    if (!ok) return;
+                    tc_fence_after();
+                    const uint32_t idesc = instr_desc(16u * (uint32_t)tile_pages(j), 0);
+                    const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
+                    const uint32_t qbase = sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u);
+                    const uint32_t kbase = sbase + kOffRing + s * kTileBytes;
 #pragma unroll
-                        for (int ks = 0; ks < kD / 16; ++ks) {
-                            const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                            mma_f16(d, smem_desc(qbase + off, 16, 1024), smem_desc(kbase + off, 16, 1024), idesc, ks > 0);
-                        }
-                        mma_commit(bar(kSFull0 + 2 * b));
-                        if (b) { ++cnt1; ++local1; } else { ++cnt0; ++local0; }
+                    for (int ks = 0; ks < kD / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                        mma_f16(d, smem_desc(qbase + off, 16, 1024), smem_desc(kbase + off, 16, 1024), idesc, ks > 0);
                     }
-                    if (ok) mma_commit(bar(kRingEmpty0 + s));
+                    mma_commit(bar(kSFull0 + 2 * b));
+                    if (release_k) mma_commit(bar(kRingEmpty0 + s));
+                };
+                // O[b] (+)= P[b] V_j with P[b] in tensor memory; fresh: first P V of the item into O[b]
+                auto issue_pv = [&](int j, int b, bool fresh, bool release_v) {
+                    const int pos = ring_pos_v(gt + j), s = pos % kRing;
+                    ok = mbar_wait(bar(kPFull0 + 2 * b), (uint32_t)(b ? cnt1 : cnt0) & 1u, abort_flag, p.status, 26) &&
+                         mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
+                    if (!ok) return;
+                    tc_fence_after();
+                    const int npg = tile_pages(j);
+                    const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b;
+                    for (int ks = 0; ks < npg; ++ks)
+                        mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks,
+                                   smem_desc(sbase + kOffRing + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
+                                   idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
+                    mma_commit(bar(kPvDone0 + 2 * b));
+                    if (b) ++cnt1; else ++cnt0;
+                    if (release_v) mma_commit(bar(kRingEmpty0 + s));
+                };
+                if (dual) {
+                    // both groups on every tile: group b owns row tile b
+                    if (ok) issue_qk(0, 0, false);
+                    if (ok) issue_qk(0, 1, true);
+                    for (int j = 0; j < ntiles && ok; ++j)
+                        for (int b = 0; b < 2 && ok; ++b) {
+                            issue_pv(j, b, j == 0, b == 1);
+                            if (ok && j + 1 < ntiles) issue_qk(j + 1, b, b == 1);
+                        }
+                } else {
+                    // one row tile: the groups take alternate KV tiles
+                    if (ok) issue_qk(0, 0, true);
+                    if (ok && ntiles > 1) issue_qk(1, 1, true);
+                    for (int j = 0; j < ntiles && ok; ++j) {
+                        issue_pv(j, j & 1, j < 2, true);
+                        if (ok && j + 2 < ntiles) issue_qk(j + 2, j & 1, true);
+                    }
                 }
                 gt += ntiles;
             }
@@ -401,51 +439,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             mma_commit(bar(kMmaDrain));
             const long long t0 = clock64();
             while (!mbar_try_wait(bar(kMmaDrain), 0) && clock64() - t0 < kWaitCycles) {}
-        }
-        __syncwarp();
-      } else if (warp == kMmaWarpPV) {
-        // ------------------------------------------------------------------ P V issuer
-        if (lane == 0) {
-            bool ok = true;
-            int gt = 0;
-            int cnt0 = 0, cnt1 = 0;
-            int item_no = 0;
-            const uint32_t idesc_pv = instr_desc(128, 1);
-            TItem it_next = load_titem(head_work, i0 < i1);
-            for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
-                const TItem it = it_next;
-                it_next = load_titem(p.works + ii + 1, ii + 1 < i1);
-                const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
-                const bool dual = it.ntok * G > kTile;
-                // O[b] (+)= P V: P (tensor memory) comes from group b, V from the ring; the first P V into
-                // an accumulator of an item overwrites it, so the previous item's epilogue must be done
-                if (item_no > 0) ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 25);
-                int first0 = 1, first1 = 1;
-                for (int j = 0; j < ntiles && ok; ++j) {
-                    const int pos = ring_pos_v(gt + j), s = pos % kRing;
-                    ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
-                    const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
-                    for (int b = dual ? 0 : (j & 1); b < (dual ? 2 : (j & 1) + 1) && ok; ++b) {
-                        const int u = b ? cnt1 : cnt0;
-                        ok = mbar_wait(bar(kPFull0 + 2 * b), (uint32_t)u & 1u, abort_flag, p.status, 26);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const bool fresh = b ? first1 : first0;
-                        const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b;
-                        for (int ks = 0; ks < npg; ++ks)
-                            mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks,
-                                       smem_desc(sbase + kOffRing + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
-                                       idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
-                        if (b) { first1 = 0; ++cnt1; } else { first0 = 0; ++cnt0; }
-                        mma_commit(bar(kPvDone0 + 2 * b));
-                    }
-                    if (ok) mma_commit(bar(kRingEmpty0 + s));
-                }
-                gt += ntiles;
-            }
-            mma_commit(bar(kMmaDrain + 1));
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bar(kMmaDrain + 1), 0) && clock64() - t0 < kWaitCycles) {}
         }
         __syncwarp();
       }

@@ -246,8 +246,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             const int ntiles = (cur.kv_end - cur.kv0 + kTileTok - 1) / kTileTok;
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
-                if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
-                else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
                 const int t1 = min(t0 + kGroupTiles, ntiles);
                 for (int t = t0; t < t1; ++t, ++n) {
                     const int s = n % S;
@@ -278,6 +276,12 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                     if (first && lane == 31) {
                         const __nv_bfloat16* src = q + ((size_t)cur.q_row0 * Hq + (size_t)cur.kv_head * GT) * D;
                         bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
+                    }
+                    // page ids of the next group of tiles (or of the next item), requested only after this
+                    // group's first tile is on its way: the next item's descriptor may still be in flight
+                    if (t == t0) {
+                        if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
+                        else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
                     }
                 }
                 pages_cur = pages_nxt;

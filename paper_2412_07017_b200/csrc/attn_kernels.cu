@@ -51,6 +51,10 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
     uint8_t* smem = aligned_smem(smem_raw);
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
     const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
+    // bring the whole header and the tensor map close now: the decode phase of a CTA that starts with
+    // span tiles finds them in L2 when it gets there
+    if (threadIdx.x < 3) asm volatile("prefetch.global.L2 [%0];" ::"l"(head + 32 * threadIdx.x));
+    if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map));
     if (head[0] == head[1]) {
         // no span tiles for this CTA: straight to its decode rows, without the tensor-memory set-up
         pdl_wait();

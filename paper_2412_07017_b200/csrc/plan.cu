@@ -218,9 +218,9 @@ struct PathCost {
     int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
 };
 // (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
-constexpr PathCost kTensorCost{128, 1530, 6200, 5700};
-constexpr PathCost kCudaCost{96, 1290, 900, 4100};
-constexpr int64_t kTensorDualTileNs = 3130;   // a KV tile of an item with two row tiles (more than 128 rows)
+constexpr PathCost kTensorCost{128, 1170, 8000, 11800};
+constexpr PathCost kCudaCost{96, 1280, 1200, 5000};
+constexpr int64_t kTensorDualTileNs = 2435;   // a KV tile of an item with two row tiles (more than 128 rows)
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
 // then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
