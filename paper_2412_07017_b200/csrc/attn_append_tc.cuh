@@ -501,7 +501,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             it_next = load_titem(p.works + ii + 1, ii + 1 < i1);
             const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
             float m_ref = -INFINITY;                     // reference maximum (log2 domain)
-            float2 l2 = make_float2(0.f, 0.f);           // running sum of P, two partial sums
+            float2 l2 = make_float2(0.f, 0.f), l2b = make_float2(0.f, 0.f);      // running sum of P, four partial sums
             int mine = 0;                                // tiles of this group so far in this item
             for (int j = dual ? 0 : b; j < ntiles && ok; j += dual ? 1 : 2, ++mine) {
                 const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
@@ -533,11 +533,20 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                             if (2 * e + 1 >= vis) x[e].y = -INFINITY;
                         }
                     }
+                    // row maximum of the half: four independent chains of 3-input maxima (a lone warp per
+                    // scheduler cannot hide one long dependent chain)
                     auto xv = [&](int k) { return (k & 1) ? x[k >> 1].y : x[k >> 1].x; };
-                    float cmax = fmax3(xv(0), xv(1), xv(2));
+                    float cm[4];
 #pragma unroll
-                    for (int k = 3; k < 63; k += 2) cmax = fmax3(cmax, xv(k), xv(k + 1));
-                    cmax = fmaxf(cmax, xv(63));
+                    for (int c = 0; c < 4; ++c) cm[c] = fmax3(xv(16 * c), xv(16 * c + 1), xv(16 * c + 2));
+#pragma unroll
+                    for (int k = 3; k < 15; k += 2) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) cm[c] = fmax3(cm[c], xv(16 * c + k), xv(16 * c + k + 1));
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) cm[c] = fmaxf(cm[c], xv(16 * c + 15));
+                    const float cmax = fmax3(fmaxf(cm[0], cm[1]), cm[2], cm[3]);
                     // x is relative to m_ref (to 0 while the row has no reference yet: then any visible key sets it)
                     if (__any_sync(0xffffffffu, cmax > (m_ref == -INFINITY ? -INFINITY : kRescaleThreshold))) {
                         // Move the reference maximum (rare after the first tile): rescale the running sum, the
@@ -548,6 +557,8 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                         m_ref = m_new;
                         l2.x *= scale;
                         l2.y *= scale;
+                        l2b.x *= scale;
+                        l2b.y *= scale;
                         const float2 ns2 = make_float2(-shift, -shift);
 #pragma unroll
                         for (int e = 0; e < 32; ++e) x[e] = __fadd2_rn(x[e], ns2);
@@ -583,7 +594,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const float2 pe = make_float2(fast_exp2(x[e].x), fast_exp2(x[e].y));
-                        l2 = __fadd2_rn(l2, pe);
+                        if (e & 1) l2b = __fadd2_rn(l2b, pe); else l2 = __fadd2_rn(l2, pe);
                         pk[e] = pack_bf16x2(pe.x, pe.y);
                     }
                     tmem_st16(s_addr + 32u * (uint32_t)h, *reinterpret_cast<uint32_t(*)[16]>(&pk[0]));
@@ -594,7 +605,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 mbar_arrive(bar(kPFull0 + 2 * b));
             }
             if (!ok) break;
-            const float l_sum = l2.x + l2.y;
+            const float l_sum = (l2.x + l2.y) + (l2b.x + l2b.y);
             load_q(it_next, q_next);        // in flight during the epilogue
             // ---- epilogue.  The groups' (max, sum) go through columns 0-1 of their S buffers, which are
             // idle from the group's last P V until the next item's first Q K^T.
