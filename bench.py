@@ -33,7 +33,7 @@ WORKLOAD = "config2-llama3-8b-mixed-batch"       # the configuration the metric 
 WORKLOADS = {2: WORKLOAD, 3: "config3-large-batch-gqa8", 4: "config4-long-context-split-kv"}
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on this workload
 # (profiles/attn_fused_kernel_config2.md); None whenever the kernel has changed since that capture
-TRAFFIC_BYTES_PER_LAUNCH = 327_289_856
+TRAFFIC_BYTES_PER_LAUNCH = 328_686_592
 
 
 def measured_peaks():
@@ -265,6 +265,18 @@ def run_gpu(args):
     torch.cuda.synchronize()
     t_wall1 = time.time()
     attn_ms = np.array([e[0].elapsed_time(e[1]) for e in ev2])
+    # Pass 3 (context only): no flush between steps.  The pool is larger than L2, so most K/V still
+    # comes from DRAM, but the kernels' code and the plan stay cached, as they do between the layers
+    # of a model; the reported value stays the flushed one.
+    ev3 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    for k in range(args.steps):
+        ev3[k][0].record(stream)
+        B.asynclm_kv_append(plan, kn, vn, pool, stream)
+        B.asynclm_attn_mixed(plan, q, pool, out, None, stream)
+        ev3[k][1].record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    noflush_ms = np.array([e[0].elapsed_time(e[1]) for e in ev3])
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
     assert B.last_device_status(plan) == 0
 
@@ -326,6 +338,7 @@ def run_gpu(args):
             "kv_tokens": int(plan.info["total_kv_tokens"]), "replicas": world,
             "l2": "256 MiB buffer rewritten between timed steps (untimed)",
             "us_per_step": ms_per_step * 1e3,
+            "us_per_step_without_l2_flush": float(np.median(noflush_ms)) * 1e3,
             "us_per_step_p10_p50_p90": [float(np.percentile(step_ms, p)) * 1e3 for p in (10, 50, 90)],
             "algorithmic_bytes_per_step": by["total"], "algorithmic_flops_per_step": flops,
             "step_hbm_frac_of_" + peak_kind: by["total"] / (ms_per_step * 1e-3) / 1e9 / peak,

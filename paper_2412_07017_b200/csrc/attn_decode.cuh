@@ -192,6 +192,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
     const int warp = threadIdx.x >> 5;
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), mbar0 = smem_u32(bars + 2 * S);
 
+    if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(kv_map));
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(full0 + 8 * s, 1);
@@ -241,6 +242,9 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         bool ok = true;
         PItem cur = load_item(i0), nxt = load_item(i0 + 1);
         int pages_cur = head[kHeadPagesCuda + lane];
+        // The plan was uploaded before the kernel in front of this one started, so all of the above
+        // overlaps that kernel's tail; the pool and Q are read only from here on.
+        pdl_wait();
         for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
             const PItem after = load_item(ii + 2);
             const int ntiles = (cur.kv_end - cur.kv0 + kTileTok - 1) / kTileTok;
@@ -309,6 +313,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
     }
 
     // ---------------------------------------------------------------------- consumer warps
+    pdl_wait();      // outputs may be written only after the kernel in front has completed
     if constexpr (FUSED) {
         if (warp < 8) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
         else asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));

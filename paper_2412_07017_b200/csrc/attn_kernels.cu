@@ -28,7 +28,6 @@ __global__ void __launch_bounds__(dec::kThreads, 1)
 attn_decode_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const __nv_bfloat16* __restrict__ q,
                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
     extern __shared__ uint8_t smem_raw[];
-    pdl_wait();
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
     dec::decode_body<D, G, false>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw));
 }
@@ -57,7 +56,6 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
     if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map));
     if (head[0] == head[1]) {
         // no span tiles for this CTA: straight to its decode rows, without the tensor-memory set-up
-        pdl_wait();
         dec::decode_body<tc::kD, G, false>(p, &kv_map, q, out, lse, S, smem);
         return;
     }
