@@ -371,6 +371,91 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_replay(args):
+    """Config 5: the interrupt-trace replay.  Every step of the trace is planned on the host, appended
+    and attended in order (the KV pool grows as the trace goes on); one untimed pass over the trace
+    warms up (re-running the appends rewrites the same bytes), the second pass is timed per step."""
+    import torch
+    from paper_2412_07017_b200 import binding as B
+    from paper_2412_07017_b200 import workload as W
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = W.make_config(5)
+    shape = wl.shape
+    steps = wl.steps[:max(1, min(args.steps, len(wl.steps)))]
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    pool = dev(wl.kv_pool)
+    dq = [(dev(st.q), dev(st.k_new), dev(st.v_new)) for st in steps]
+    max_T = max(st.total_q for st in steps)
+    out = torch.empty((max_T, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    hb, db = B.workspace_size(shape, wl.num_pages, steps[0].batch, max_T,
+                              max(len(st.page_indices) for st in steps))
+    host_ws = torch.empty(hb, dtype=torch.uint8).pin_memory()
+    dev_ws = torch.empty(db, dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(0)
+    plan_us, dev_us, kv_bytes, tot_bytes, spans = [], [], [], [], []
+    launches = 0
+    for timed in (False, True):
+        t_wall0 = time.time()
+        for k, st in enumerate(steps):
+            t0 = time.perf_counter()
+            plan = B.asynclm_plan(shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr,
+                                  st.page_indices, host_ws=host_ws, dev_ws=dev_ws)
+            t1 = time.perf_counter()
+            flush.fill_(k & 0xff)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            B.asynclm_kv_append(plan, dq[k][1], dq[k][2], pool, stream)
+            B.asynclm_attn_mixed(plan, dq[k][0], pool, out, None, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()          # the plan workspaces are reused by the next step
+            assert B.last_device_status(plan) == 0
+            if timed:
+                by = W.algorithmic_bytes(shape, st)
+                plan_us.append((t1 - t0) * 1e6)
+                dev_us.append(e0.elapsed_time(e1) * 1e3)
+                kv_bytes.append(by["kv"])
+                tot_bytes.append(by["total"])
+                spans.append(int((st.q_len > 1).sum()))
+                launches += plan.info["launches_append"] + plan.info["launches_attn"]
+        t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    peak, peak_kind = measured_peaks()
+    dev_us = np.array(dev_us)
+    total_s = float(dev_us.sum()) * 1e-6
+    line = {
+        "metric": METRIC, "value": float(np.sum(kv_bytes)) / total_s / 1e9, "unit": UNIT, "n_gpus": 1,
+        "steps": len(steps), "warmup": len(steps), "ms_per_step": float(dev_us.mean()) * 1e-3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": "config5-interrupt-trace-replay", "seed": wl.seed, "batch": steps[0].batch,
+            "l2": "256 MiB buffer rewritten between timed steps (untimed)",
+            "us_per_step_first_median_last": [float(dev_us[0]), float(np.median(dev_us)), float(dev_us[-1])],
+            "us_per_step_p10_p90": [float(np.percentile(dev_us, 10)), float(np.percentile(dev_us, 90))],
+            "us_per_step_with_interrupts": float(dev_us[np.array(spans) > 0].mean()) if any(spans) else None,
+            "us_per_step_decode_only": float(dev_us[np.array(spans) == 0].mean()) if not all(spans) else None,
+            "steps_with_interrupts": int((np.array(spans) > 0).sum()),
+            "kv_mb_first_last": [kv_bytes[0] / 1e6, kv_bytes[-1] / 1e6],
+            "plan_host_us_median": float(np.median(plan_us)),
+            "step_hbm_frac_of_" + peak_kind: float(np.sum(tot_bytes)) / total_s / 1e9 / peak,
+        },
+        "roofline": {"bound": "hbm", "kernel": "whole step (append + attention + merge), all trace steps",
+                     "achieved": float(np.sum(tot_bytes)) / total_s / 1e9, "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": float(np.sum(tot_bytes)) / total_s / 1e9 / peak, "traffic": None},
+        "e2e": {"value": float(np.sum(kv_bytes)) / (total_s + float(np.sum(plan_us)) * 1e-6) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                "includes": "asynclm_plan on the host (+ its upload) and the device step; inputs resident"},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -378,13 +463,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
-                    help="synthetic configuration; 2 is the benchmark, 3 and 4 are for reference")
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5],
+                    help="synthetic configuration; 2 is the benchmark, 3 and 4 are for reference, "
+                         "5 replays the interrupt trace step by step")
     ap.add_argument("--decode-only", action="store_true",
                     help="time a decode-only batch instead (exercises attn_decode_kernel alone)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == 5:
+        run_replay(args)
     else:
         run_gpu(args)
 

@@ -257,6 +257,8 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     auto fill = [&](int64_t cap, std::vector<Piece> (&out)[2]) {
         out[0].clear();
         out[1].clear();
+        out[0].reserve(ids_tensor.size() + (size_t)n_ctas);
+        out[1].reserve(ids_cuda.size() + (size_t)n_ctas);
         bool fits = true;
         std::vector<int64_t> load((size_t)n_ctas, 0);
         int used = 0;                                   // CTAs that hold span work: [0, used)
@@ -333,7 +335,7 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     // Smallest limit that fits, by bisection (the loads are monotone in the limit up to rounding).
     int64_t lo = std::max<int64_t>(1, total / n_ctas), hi = 2 * lo + kTensorCost.item_ns + kTensorCost.phase_ns + kCudaCost.phase_ns;
     while (!fill(hi, best)) hi *= 2;
-    for (int iter = 0; iter < 24 && hi - lo > 50; ++iter) {
+    for (int iter = 0; iter < 24 && hi - lo > std::max<int64_t>(50, hi / 256); ++iter) {      // to 0.4 %
         const int64_t mid = (lo + hi) / 2;
         std::vector<Piece> trial[2];
         if (fill(mid, trial)) {
