@@ -44,7 +44,7 @@ namespace asynclm {
 namespace tc {
 
 constexpr int kThreads = 384;
-constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10, kMmaWarpPV = 11;
+constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10;      // warp 11 idles
 constexpr int kD = 128;
 constexpr int kTile = 128;                       // keys per K/V ring slot and query rows per row tile
 constexpr int kSub = 64;                         // keys the softmax handles at a time (half an S tile)
@@ -61,7 +61,7 @@ constexpr uint32_t kOffBar = kOffRing + kRing * kTileBytes;
 // S, P V and P hand-offs exist per group b: index 2 * b
 enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPvDone0 = kPFull0 + 4, kSFull0 = kPvDone0 + 4,
            kRingFull0 = kSFull0 + 4, kRingEmpty0 = kRingFull0 + kRing, kMmaDrain = kRingEmpty0 + kRing,
-           kMmaDrain2, kNumBars };
+           kNumBars };
 constexpr uint32_t kOffTmemPtr = kOffBar + 8 * kNumBars;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
 constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
@@ -271,7 +271,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         }
         for (int s = 0; s < kRing; ++s) { mbar_init(bar(kRingFull0 + s), 32); mbar_init(bar(kRingEmpty0 + s), 1); }
         mbar_init(bar(kMmaDrain), 1);
-        mbar_init(bar(kMmaDrain + 1), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
