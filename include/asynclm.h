@@ -74,8 +74,8 @@ typedef struct asynclm_plan_options {
                                  the work items roughly fill the machine; a value >= the longest
                                  context disables splitting */
     int32_t tensor_min_rows;  /* a span uses the tensor-core path when G * q_len >= this;
-                                 0 = default; a value > 128*G*... (INT32_MAX) keeps every row on
-                                 the CUDA-core path */
+                                 0 = default (32); INT32_MAX keeps every row on the CUDA-core
+                                 path, like ASYNCLM_PLAN_NO_TENSOR_PATH */
     int32_t flags;            /* ASYNCLM_PLAN_* */
 } asynclm_plan_options;
 
@@ -148,8 +148,9 @@ int asynclm_plan_workspace_size(const asynclm_shape* shape, const asynclm_plan_o
  *
  * Validates the batch, tiles every (sequence, kv head) into query tiles and page-aligned KV chunks
  * (long contexts are split; partial results are merged by log-sum-exp inside asynclm_attn_mixed),
- * orders the items longest-first and assigns them to persistent CTAs, then enqueues ONE
- * host->device copy of the packed plan on `stream`.
+ * assigns the items to persistent CTAs under the smallest per-CTA load limit that fits (span tiles
+ * are kept whole where possible, largest first; decode rows fill the CTAs up and are cut only
+ * where a CTA is full), then enqueues ONE host->device copy of the packed plan on `stream`.
  *
  *   host_ws / host_bytes  host memory (8-byte aligned; pinned recommended) that must stay untouched
  *                         until the copy has completed and for as long as the plan is used.

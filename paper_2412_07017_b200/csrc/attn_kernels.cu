@@ -2,7 +2,8 @@
 //
 // Three kernels are built from two bodies (attn_append_tc.cuh: tensor-core span tiles,
 // attn_decode.cuh: CUDA-core decode rows):
-//   attn_fused_kernel      a persistent CTA first runs its tensor-core items, then its CUDA-core items.
+//   attn_fused_kernel      a persistent CTA first runs its tensor-core items, then its CUDA-core items
+//                          (a CTA without span tiles skips the tensor-memory set-up altogether).
 //                          One launch instead of two: the fixed cost of a launch (about 10 us of
 //                          start-up and tail per kernel at 148 CTAs) is paid once, and a CTA that is
 //                          done with its span tiles early moves on to decode rows at once.

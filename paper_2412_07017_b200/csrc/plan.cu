@@ -223,10 +223,9 @@ constexpr PathCost kCudaCost{96, 1280, 1200, 5000};
 constexpr int64_t kTensorDualTileNs = 2435;   // a KV tile of an item with two row tiles (more than 128 rows)
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
-// then its CUDA-core items: all units are laid on one line (tensor units first), weighted with the
-// measured costs, and the line is cut into n_ctas nearly equal pieces.  A unit is split only where a
-// piece boundary falls inside it, so there are at most n_ctas - 1 more items than units, most CTAs
-// run one kind of work only, and the two kinds finish together.
+// then its CUDA-core items: units are weighted with the measured costs and dealt under a per-CTA load
+// limit (see `fill` below); the smallest limit that fits is found by bisection, so that all CTAs
+// finish together as far as the cost model holds.
 void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& ids_cuda,
                   std::vector<UnitBuild>& units, int group, int n_ctas, std::vector<Item>& items,
                   std::vector<int32_t>& cta_indptr_cuda, std::vector<int32_t>& cta_indptr_tensor,
