@@ -147,3 +147,60 @@ def test_workspace_size_bounds_actual_use():
     hb, db = B.workspace_size(wl.shape, wl.num_pages, st.batch, st.total_q, len(st.page_indices),
                               num_sms=148, kv_chunk_tokens=64)
     assert hb >= p.info["host_bytes_used"] and db >= p.info["device_bytes_used"]
+
+
+def _llama_lengths(seed=0):
+    g = np.random.default_rng(seed)
+    ctx = g.integers(512, 4097, 32)
+    ql = np.ones(32, dtype=np.int64)
+    ql[:8] = g.integers(8, 65, 8)
+    need = -(-(ctx + ql) // 16)
+    q_indptr, page_indptr, page_indices, _ = W.build_step_tables(ctx, ql, 16, np.arange(need.sum()))
+    return ctx, ql, int(need.sum()), q_indptr, page_indptr, page_indices
+
+
+def test_mixed_batch_spans_stay_whole_and_loads_balance():
+    """Default policy on the Llama-shaped mixed batch: every (token, key) pair is covered once, span
+    units are cut only when one is larger than a CTA's share, cuts fall on tile boundaries, and the
+    CTAs' tile counts are balanced."""
+    ctx, ql, num_pages, q_indptr, page_indptr, page_indices = _llama_lengths()
+    shape = W.Shape(32, 8, 128, 16)
+    p = B.plan_host(shape, num_pages, q_indptr, ctx, page_indptr, page_indices, num_sms=148)
+    items = p.items()
+    # coverage, per (sequence, kv head, token)
+    for b in range(32):
+        for h in (0, 7):
+            for i in {0, int(ql[b]) - 1}:
+                segs = sorted((int(it["kv0"]), min(int(it["kv1"]), int(ctx[b]) + i + 1)) for it in items
+                              if it["seq"] == b and it["kv_head"] == h and it["tok0"] <= i < it["tok0"] + it["ntok"])
+                segs = [s for s in segs if s[1] > s[0]]
+                assert segs[0][0] == 0 and segs[-1][1] == int(ctx[b]) + i + 1
+                assert all(a[1] == c[0] for a, c in zip(segs[:-1], segs[1:]))
+    span = items[items["path"] == 1]
+    dec = items[items["path"] == 0]
+    assert len(span) and len(dec)
+    assert (span["kv0"] % 128 == 0).all() and (dec["kv0"] % 96 == 0).all()
+    # a span unit covers up to 256 (token, head) rows: 64 tokens at 4 heads per kv head
+    assert span["ntok"].max() <= 64 and (span["tok0"] % 64 == 0).all()
+    units = {(int(it["seq"]), int(it["kv_head"]), int(it["tok0"])) for it in span}
+    pieces = len(span) / len(units)
+    assert pieces < 1.6, pieces          # most span units are one item (no partial rows, no merge)
+    # modelled load per CTA in KV tiles (a span tile of two row tiles counts double)
+    load = np.zeros(148)
+    np.add.at(load, span["cta"], -(-(span["kv1"] - span["kv0"]) // 128) * np.where(span["ntok"] * 4 > 128, 2.0, 1.0))
+    np.add.at(load, dec["cta"], -(-(dec["kv1"] - dec["kv0"]) // 96))
+    assert load.max() <= 1.35 * load.mean()
+    assert p.info["launches_attn"] == 2 and p.info["num_split_units"] > 0
+
+
+def test_decode_only_batch_has_no_span_items():
+    ctx, ql, num_pages, q_indptr, page_indptr, page_indices = _llama_lengths(1)
+    ql[:] = 1
+    need = -(-(ctx + ql) // 16)
+    q_indptr, page_indptr, page_indices, _ = W.build_step_tables(ctx, ql, 16, np.arange(need.sum()))
+    p = B.plan_host(W.Shape(32, 8, 128, 16), int(need.sum()), q_indptr, ctx, page_indptr, page_indices, num_sms=148)
+    items = p.items()
+    assert (items["path"] == 0).all() and p.info["num_items_tensor"] == 0
+    load = np.zeros(148)
+    np.add.at(load, items["cta"], -(-(items["kv1"] - items["kv0"]) // 96))
+    assert load.max() <= 1.15 * load.mean() + 1
