@@ -248,33 +248,48 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     // it, else into a fresh CTA; a unit larger than a CTA's share is cut into equal pieces.
     //   Decode units then fill every CTA up to the limit in CTA order; a unit is cut only where a
     // CTA is full.
+    //   With emit == false only the verdict is computed (the bisection's probes).
     std::vector<int> tensor_order(ids_tensor);
-    auto unit_tiles = [&](int path, int id) { return (units[id].n_keys + cost[path].gran - 1) / cost[path].gran; };
+    std::vector<int64_t> tiles_of(units.size()), tns_of(units.size());
+    for (int path = 0; path < 2; ++path)
+        for (int id : *ids[path]) {
+            tiles_of[(size_t)id] = (units[id].n_keys + cost[path].gran - 1) / cost[path].gran;
+            tns_of[(size_t)id] = tile_ns(path, id);
+        }
+    auto unit_tiles = [&](int, int id) { return tiles_of[(size_t)id]; };
     std::stable_sort(tensor_order.begin(), tensor_order.end(), [&](int x, int y) {
-        return unit_tiles(0, x) * tile_ns(0, x) > unit_tiles(0, y) * tile_ns(0, y);
+        return tiles_of[(size_t)x] * tns_of[(size_t)x] > tiles_of[(size_t)y] * tns_of[(size_t)y];
     });
-    auto fill = [&](int64_t cap, std::vector<Piece> (&out)[2]) {
+    std::vector<int64_t> load((size_t)n_ctas);
+    auto fill = [&](int64_t cap, std::vector<Piece> (&out)[2], bool emit) {
         out[0].clear();
         out[1].clear();
-        out[0].reserve(ids_tensor.size() + (size_t)n_ctas);
-        out[1].reserve(ids_cuda.size() + (size_t)n_ctas);
+        if (emit) {
+            out[0].reserve(ids_tensor.size() + (size_t)n_ctas);
+            out[1].reserve(ids_cuda.size() + (size_t)n_ctas);
+        }
         bool fits = true;
-        std::vector<int64_t> load((size_t)n_ctas, 0);
+        std::fill(load.begin(), load.end(), (int64_t)0);
         int used = 0;                                   // CTAs that hold span work: [0, used)
+        int64_t least = INT64_MAX;                      // lower bound of the smallest load among them
         {
             const PathCost& pc = cost[0];
+            // tiles a fresh CTA takes, for the two kinds of span tile
+            const int64_t fresh_single = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / pc.tile_ns);
+            const int64_t fresh_dual = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / kTensorDualTileNs);
             for (int id : tensor_order) {
-                const int64_t tns = tile_ns(0, id);
+                const int64_t tns = tns_of[(size_t)id];
                 const int64_t tiles = unit_tiles(0, id);
-                const int64_t fresh_room = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / tns);   // tiles a fresh CTA takes
-                const int64_t pieces = (tiles + fresh_room - 1) / fresh_room;
+                const int64_t fresh_room = tns == pc.tile_ns ? fresh_single : fresh_dual;
+                const int64_t pieces = tiles <= fresh_room ? 1 : (tiles + fresh_room - 1) / fresh_room;
                 int64_t k0 = 0;
                 for (int64_t c = 0; c < pieces; ++c) {
-                    const int64_t take = tiles / pieces + (c < tiles % pieces ? 1 : 0);
+                    const int64_t take = pieces == 1 ? tiles : tiles / pieces + (c < tiles % pieces ? 1 : 0);
                     const int64_t need = pc.item_ns + take * tns;
                     int best_cta = -1;
-                    for (int k = 0; k < used; ++k)
-                        if (load[(size_t)k] + need <= cap && (best_cta < 0 || load[(size_t)k] > load[(size_t)best_cta])) best_cta = k;
+                    if (least + need <= cap)            // otherwise no span CTA has room: skip the scan
+                        for (int k = 0; k < used; ++k)
+                            if (load[(size_t)k] + need <= cap && (best_cta < 0 || load[(size_t)k] > load[(size_t)best_cta])) best_cta = k;
                     if (best_cta < 0) {
                         if (used < n_ctas) {
                             best_cta = used++;
@@ -286,8 +301,10 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
                         }
                     }
                     const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
-                    out[0].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c}, (int32_t)best_cta});
+                    if (emit) out[0].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c}, (int32_t)best_cta});
+                    else if (!fits) return false;
                     load[(size_t)best_cta] += need;
+                    least = std::min(least, load[(size_t)best_cta]);
                     k0 = k1;
                 }
             }
@@ -319,7 +336,8 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
                         take = std::max<int64_t>(1, room / pc.tile_ns);
                     }
                     const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
-                    out[1].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
+                    if (emit) out[1].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
+                    else if (!fits) return false;
                     load[(size_t)cta] += start + take * pc.tile_ns;
                     has_phase = true;
                     left -= take;
@@ -332,19 +350,15 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
         return fits;
     };
     // Smallest limit that fits, by bisection (the loads are monotone in the limit up to rounding).
-    int64_t lo = std::max<int64_t>(1, total / n_ctas), hi = 2 * lo + kTensorCost.item_ns + kTensorCost.phase_ns + kCudaCost.phase_ns;
-    while (!fill(hi, best)) hi *= 2;
-    for (int iter = 0; iter < 24 && hi - lo > std::max<int64_t>(50, hi / 256); ++iter) {      // to 0.4 %
+    // The probes only ask whether a limit fits; the pieces are built once, for the limit found.
+    int64_t lo = std::max<int64_t>(1, total / n_ctas);
+    int64_t hi = lo + lo / 4 + kTensorCost.item_ns + kTensorCost.phase_ns + kCudaCost.phase_ns;
+    while (!fill(hi, best, false)) { lo = hi; hi += hi / 2; }
+    for (int iter = 0; iter < 24 && hi - lo > std::max<int64_t>(50, hi / 128); ++iter) {      // to 0.8 %
         const int64_t mid = (lo + hi) / 2;
-        std::vector<Piece> trial[2];
-        if (fill(mid, trial)) {
-            hi = mid;
-            best[0].swap(trial[0]);
-            best[1].swap(trial[1]);
-        } else {
-            lo = mid;
-        }
+        if (fill(mid, best, false)) hi = mid; else lo = mid;
     }
+    fill(hi, best, true);
     // emit: CUDA-core items first, then tensor items; chunk counts per unit
     cta_indptr_cuda.assign((size_t)n_ctas + 1, 0);
     cta_indptr_tensor.assign((size_t)n_ctas + 1, 0);
