@@ -19,8 +19,9 @@
 //                   writes P as packed bf16 pairs over the columns it has already read; P V then
 //                   takes its A operand from tensor memory.  The reference maximum only moves when
 //                   a score exceeds it by 2^8; then O, the running sum and the half of P already
-//                   written are rescaled.  The exponentials bound this stage (16 per clock and SM),
-//                   so everything around them is packed two values to an instruction.
+//                   written are rescaled.  With one softmax warp per scheduler the stage is bound
+//                   by issue slots and dependent latency, so the arithmetic around the exponentials
+//                   is packed two values to an instruction and reductions run in independent chains.
 //                   At the end of an item the rows go out through the group's (now idle) Q tile in
 //                   shared memory, so that every global store writes whole 128-byte lines.
 //   warps 8, 10     producers of K tiles and of V tiles: 16-byte cp.async copies (fully coalesced,
