@@ -233,7 +233,13 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     struct Piece { Item it; int32_t cta; };
     std::vector<Piece> best[2];
     const std::vector<int>* ids[2] = {&ids_tensor, &ids_cuda};
-    const PathCost cost[2] = {kTensorCost, kCudaCost};
+    PathCost cost[2] = {kTensorCost, kCudaCost};
+    if (group > 4) {
+        // 8 heads per kv head: the decode kernel runs two head halves over 48-key tiles and is bound by
+        // its arithmetic; measured 2.42 us per 96 keys and 1.4 us per item on the 64/8-head batch
+        cost[1].tile_ns = 2420;
+        cost[1].item_ns = 1400;
+    }
     auto tile_ns = [&](int path, int id) {
         return path == 0 && units[id].u.ntok * group > 128 ? kTensorDualTileNs : cost[path].tile_ns;
     };
