@@ -73,9 +73,12 @@ typedef struct asynclm_plan_options {
     int32_t kv_chunk_tokens;  /* fixed split-KV chunk length (multiple of 64); 0 = chosen so that
                                  the work items roughly fill the machine; a value >= the longest
                                  context disables splitting */
-    int32_t tensor_min_rows;  /* a span uses the tensor-core path when G * q_len >= this;
-                                 0 = default (32); INT32_MAX keeps every row on the CUDA-core
-                                 path, like ASYNCLM_PLAN_NO_TENSOR_PATH */
+    int32_t tensor_min_rows;  /* new tokens of a sequence use the tensor-core path when
+                                 G * q_len >= this; 0 = default: 32 (decode rows stay on the
+                                 CUDA-core path) for G <= 4, and 8 for G = 8, where the CUDA-core
+                                 path is bound by its arithmetic rather than by memory;
+                                 INT32_MAX keeps every row on the CUDA-core path, like
+                                 ASYNCLM_PLAN_NO_TENSOR_PATH */
     int32_t flags;            /* ASYNCLM_PLAN_* */
 } asynclm_plan_options;
 

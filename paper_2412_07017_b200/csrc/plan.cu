@@ -44,7 +44,13 @@ static int check_shape(const asynclm_shape* s) {
 // Tokens of a span that one tensor-core work item covers: two row tiles of 128 (token, head) rows.
 int tensor_tile_tokens(int group) { return 256 / group; }
 
-static int default_tensor_min_rows() { return 32; }
+// Rows (G * q_len) from which a (sequence, kv head) goes to the tensor-core kernel.  Up to 4 heads per
+// kv head a decode row stays on the CUDA-core kernel, which then runs near the memory rate, and spans
+// of 32 rows and more take the tensor cores.  With 8 heads per kv head every KV byte feeds twice the
+// arithmetic and the CUDA-core kernel is bound by its FMAs at half the memory rate (measured:
+// 2.4 TB/s against 4.1 TB/s on the 64/8-head batch), so there the 8 rows of a decode token already
+// count as wide enough.
+static int default_tensor_min_rows(int group) { return group >= 8 ? 8 : 32; }
 
 // Sizes of the sections of the packed blob (identical offsets on host and device).
 struct BlobLayout {
@@ -471,7 +477,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     const bool tensor_ok = !(opts && (opts->flags & ASYNCLM_PLAN_NO_TENSOR_PATH)) &&
                            tensor_path_compiled(shape->head_dim);
     const int tensor_min_rows =
-        (opts && opts->tensor_min_rows > 0) ? opts->tensor_min_rows : default_tensor_min_rows();
+        (opts && opts->tensor_min_rows > 0) ? opts->tensor_min_rows : default_tensor_min_rows(G);
     const int TQ = tensor_tile_tokens(G);
     std::vector<UnitBuild> units;
     std::vector<int> ids_cuda, ids_tensor;

@@ -49,10 +49,23 @@ def test_fixed_chunk_lengths_agree_with_oracle(chunk):
         assert plan.info["num_split_units"] > 0
 
 
-def test_cuda_core_path_handles_spans_too():
-    shape = W.Shape(8, 2, 128, 16)
-    wl = W.make_single_step("spans", shape, [300, 0, 40], [64, 130, 9], seed=78)
-    run_and_check(wl, what="cuda-core spans", flags=B.PLAN_NO_TENSOR_PATH)
+@pytest.mark.parametrize("Hq", [8, 16])
+def test_cuda_core_path_handles_spans_too(Hq):
+    """Every row on the CUDA-core kernel (4 and 8 heads per kv head; with 8 the planner would send
+    even decode rows to the tensor cores by default)."""
+    shape = W.Shape(Hq, 2, 128, 16)
+    wl = W.make_single_step("spans", shape, [300, 0, 40, 700], [64, 130, 9, 1], seed=78)
+    _, _, plan = run_and_check(wl, what="cuda-core spans", flags=B.PLAN_NO_TENSOR_PATH)
+    assert plan.info["num_items_tensor"] == 0
+
+
+def test_eight_heads_per_kv_head_decode_rows_take_the_tensor_path():
+    shape = W.Shape(16, 2, 128, 16)
+    wl = W.make_single_step("gqa8", shape, [300, 0, 1500, 77], [1, 1, 1, 20], seed=79)
+    _, _, plan = run_and_check(wl, what="gqa8 decode on tensor cores")
+    assert plan.info["num_items_tensor"] == plan.info["num_items"]
+    _, _, plan = run_and_check(wl, what="gqa8 decode on cuda cores", tensor_min_rows=32)
+    assert 0 < plan.info["num_items_tensor"] < plan.info["num_items"]
 
 
 def test_results_are_bitwise_reproducible():
