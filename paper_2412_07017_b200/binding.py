@@ -47,11 +47,12 @@ class CPlanOptions(ctypes.Structure):
 
 
 class CBatch(ctypes.Structure):
+    # the four arrays are `const int32_t*` in C; plain addresses marshal faster than typed pointers
     _fields_ = [("batch", ctypes.c_int32),
-                ("q_indptr", ctypes.POINTER(ctypes.c_int32)),
-                ("kv_len_before", ctypes.POINTER(ctypes.c_int32)),
-                ("page_indptr", ctypes.POINTER(ctypes.c_int32)),
-                ("page_indices", ctypes.POINTER(ctypes.c_int32))]
+                ("q_indptr", ctypes.c_void_p),
+                ("kv_len_before", ctypes.c_void_p),
+                ("page_indptr", ctypes.c_void_p),
+                ("page_indices", ctypes.c_void_p)]
 
 
 class CPlanInfo(ctypes.Structure):
@@ -127,8 +128,9 @@ def _copts(num_sms=0, kv_chunk_tokens=0, tensor_min_rows=0, flags=0) -> CPlanOpt
 
 
 def _i32(a):
-    a = np.ascontiguousarray(a, dtype=np.int32)
-    return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+    if not (isinstance(a, np.ndarray) and a.dtype == np.int32 and a.flags.c_contiguous):
+        a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data
 
 
 def _cbatch(q_indptr, kv_len_before, page_indptr, page_indices):
@@ -149,11 +151,19 @@ def workspace_size(shape, num_pages, max_batch, max_total_q, max_total_pages, **
 
 @dataclass
 class Plan:
+    """A plan handle with the workspaces it lives in.  `info` (what the planner decided) is read from
+    the plan on first access, so look at it before the workspaces are reused for another plan."""
     handle: int
-    info: dict
     host_ws: object
     dev_ws: object
     keepalive: object = None
+    _info: Optional[dict] = None
+
+    @property
+    def info(self) -> dict:
+        if self._info is None:
+            self._info = _get_info(self.handle)
+        return self._info
 
     def items(self) -> np.ndarray:
         n = self.info["num_items"]
@@ -187,7 +197,7 @@ def plan_host(shape, num_pages, q_indptr, kv_len_before, page_indptr, page_indic
             hbytes *= 4
             continue
         _check(rc, "asynclm_plan")
-        return Plan(out.value, _get_info(out.value), ws, None, keep)
+        return Plan(out.value, ws, None, keep)
 
 
 def asynclm_plan(shape, num_pages, q_indptr, kv_len_before, page_indptr, page_indices,
@@ -217,7 +227,7 @@ def asynclm_plan(shape, num_pages, q_indptr, kv_len_before, page_indptr, page_in
     _check(lib.asynclm_plan(ctypes.byref(cs), ctypes.byref(co), ctypes.byref(cb),
                             host_ws.data_ptr(), host_ws.numel(), dev_ws.data_ptr(), dev_ws.numel(),
                             s, ctypes.byref(out)), "asynclm_plan")
-    return Plan(out.value, _get_info(out.value), host_ws, dev_ws, None)
+    return Plan(out.value, host_ws, dev_ws, None)
 
 
 def _stream_ptr(stream):
