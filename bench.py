@@ -187,6 +187,11 @@ def run_gpu(args):
         # token each: the CUDA-core decode kernel alone (profiling aid, not the benchmarked workload)
         lens = np.random.default_rng(3).integers(1024, 3073, 64).tolist()
         wl = W.make_single_step("decode-only", W.Shape(32, 8, 128, 16), lens, [1] * 64, seed=11)
+    elif args.spans_only:
+        # 24 sequences of the same shape, contexts uniform in [1024, 3072], every one with an interrupt
+        # span of 64 tokens (256 query rows per kv head): the tensor-core span kernel alone
+        lens = np.random.default_rng(4).integers(1024, 3073, 24).tolist()
+        wl = W.make_single_step("spans-only", W.Shape(32, 8, 128, 16), lens, [64] * 24, seed=12)
     else:
         wl = W.make_config(args.config)
     st = wl.steps[0]
@@ -338,7 +343,9 @@ def run_gpu(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": "decode-only-64x[1024,3072]" if args.decode_only else WORKLOADS[args.config], "seed": wl.seed, "batch": st.batch, "total_q": T,
+            "workload": "decode-only-64x[1024,3072]" if args.decode_only else
+                        "spans-only-24x[1024,3072]+64" if args.spans_only else WORKLOADS[args.config],
+            "seed": wl.seed, "batch": st.batch, "total_q": T,
             "kv_tokens": int(plan.info["total_kv_tokens"]), "replicas": world,
             "l2": "256 MiB buffer rewritten between timed steps (untimed)",
             "us_per_step": ms_per_step * 1e3,
@@ -352,10 +359,11 @@ def run_gpu(args):
                                                "kv_chunk_tokens", "num_ctas_cuda", "num_ctas_tensor")},
         },
         "roofline": {"bound": "hbm",
-                     "kernel": ("attn_decode_kernel" if args.decode_only else "attn_fused_kernel") +
+                     "kernel": ("attn_decode_kernel" if args.decode_only else
+                                "attn_append_tc_kernel" if args.spans_only else "attn_fused_kernel") +
                                " (+ lse_merge_kernel; timed together as asynclm_attn_mixed)",
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.config == 2 and not args.decode_only else None,
+                     "frac": achieved / peak, "traffic": TRAFFIC_BYTES_PER_LAUNCH if args.config == 2 and not (args.decode_only or args.spans_only) else None,
                      "algorithmic_bytes_per_launch": attn_bytes, "avg_launch_us": attn_s * 1e6},
         "e2e": {"value": world * by["kv"] / (e2e_total / e2e_steps) / 1e9, "unit": UNIT,
                 "h2d_bytes_per_step": int(h2d),
@@ -472,6 +480,8 @@ def main():
                          "5 replays the interrupt trace step by step")
     ap.add_argument("--decode-only", action="store_true",
                     help="time a decode-only batch instead (exercises attn_decode_kernel alone)")
+    ap.add_argument("--spans-only", action="store_true",
+                    help="time a batch in which every sequence gets a 64-token span (attn_append_tc_kernel alone)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
