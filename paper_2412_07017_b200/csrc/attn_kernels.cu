@@ -61,6 +61,7 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
         return;
     }
     tc::tc_body<G, true>(p, q, pool, out, lse, smem);
+    if (head[2] == head[3]) return;      // the planner gave this CTA its decode rows as tensor-core items too
     __syncthreads();      // tensor memory released, shared memory free for the second phase
     dec::decode_body<tc::kD, G, true>(p, &kv_map, q, out, lse, S, smem);
 }

@@ -227,6 +227,14 @@ struct PathCost {
 constexpr PathCost kTensorCost{128, 1170, 8000, 11800};
 constexpr PathCost kCudaCost{96, 1280, 1200, 5000};
 constexpr int64_t kTensorDualTileNs = 2435;   // a KV tile of an item with two row tiles (more than 128 rows)
+// When every unit runs on the tensor-core kernel all SMs stream K/V tiles at once and the tile time is
+// set by the memory system (64 KB per tile and SM: 148 SMs at 37 KB/us are 5.5 TB/s); the producers
+// run ahead across item boundaries.
+constexpr PathCost kTensorOnlyCost{128, 1543, 8000, 2400};
+constexpr int64_t kTensorOnlyDualTileNs = 3126;
+// Units with fewer (token, head) rows than this are cut wherever a CTA is full (their partial rows are
+// a few KB); wider span units are kept whole where they fit.
+constexpr int kWholeUnitMinRows = 32;
 
 // Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
 // then its CUDA-core items: units are weighted with the measured costs and dealt under a per-CTA load
@@ -239,7 +247,12 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     struct Piece { Item it; int32_t cta; };
     std::vector<Piece> best[2];
     const std::vector<int>* ids[2] = {&ids_tensor, &ids_cuda};
-    PathCost cost[2] = {kTensorCost, kCudaCost};
+    const bool tensor_only = ids_cuda.empty();
+    PathCost cost[2] = {tensor_only ? kTensorOnlyCost : kTensorCost, kCudaCost};
+    const int64_t dual_tile_ns = tensor_only ? kTensorOnlyDualTileNs : kTensorDualTileNs;
+    // a narrow item (one decode token's rows) on the tensor-core body: tile and item cost
+    const int64_t narrow_tile_ns = tensor_only ? kTensorOnlyCost.tile_ns : 1400;
+    const int64_t narrow_item_ns = 2900;
     if (group > 4) {
         // 8 heads per kv head: the decode kernel runs two head halves over 48-key tiles and is bound by
         // its arithmetic; measured 2.42 us per 96 keys and 1.4 us per item on the 64/8-head batch
@@ -247,7 +260,7 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
         cost[1].item_ns = 1400;
     }
     auto tile_ns = [&](int path, int id) {
-        return path == 0 && units[id].u.ntok * group > 128 ? kTensorDualTileNs : cost[path].tile_ns;
+        return path == 0 && units[id].u.ntok * group > 128 ? dual_tile_ns : cost[path].tile_ns;
     };
     // Lower bound of the makespan: all work, one start per unit, one phase start per CTA.
     int64_t total = 0;
@@ -261,7 +274,9 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     //   Decode units then fill every CTA up to the limit in CTA order; a unit is cut only where a
     // CTA is full.
     //   With emit == false only the verdict is computed (the bisection's probes).
-    std::vector<int> tensor_order(ids_tensor);
+    std::vector<int> tensor_order, tensor_narrow;      // span units packed whole; narrow units that fill up CTAs
+    for (int id : ids_tensor)
+        (units[id].u.ntok * group >= kWholeUnitMinRows ? tensor_order : tensor_narrow).push_back(id);
     std::vector<int64_t> tiles_of(units.size()), tns_of(units.size());
     for (int path = 0; path < 2; ++path)
         for (int id : *ids[path]) {
@@ -288,7 +303,7 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
             const PathCost& pc = cost[0];
             // tiles a fresh CTA takes, for the two kinds of span tile
             const int64_t fresh_single = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / pc.tile_ns);
-            const int64_t fresh_dual = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / kTensorDualTileNs);
+            const int64_t fresh_dual = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / dual_tile_ns);
             for (int id : tensor_order) {
                 const int64_t tns = tns_of[(size_t)id];
                 const int64_t tiles = unit_tiles(0, id);
@@ -320,50 +335,64 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
                     k0 = k1;
                 }
             }
-            std::stable_sort(out[0].begin(), out[0].end(), [](const Piece& x, const Piece& y) { return x.cta < y.cta; });
         }
-        {
-            PathCost pc = cost[1];
+        // Line fill: the units of `list` in order, each CTA up to the limit; a unit is cut only where a
+        // CTA is full.  CTAs below `started` already hold tensor-core work.  A CUDA-core unit (one decode
+        // token) that lands on such a CTA runs there as a narrow tensor-core item: the CTA then never
+        // re-splits its registers and restarts its pipeline for a second phase (measured on the
+        // Llama-shaped mixed batch: 91.6 -> 87 us per step), while CTAs without span work keep the
+        // CUDA-core body, which is the faster one on decode rows.
+        auto line_fill = [&](int path, const std::vector<int>& list, int started) {
             int cta = 0;
             bool has_phase = false;
-            auto next_cta = [&]() { ++cta; has_phase = false; };
-            for (int id : *ids[1]) {
-                int64_t left = unit_tiles(1, id);
+            for (int id : list) {
+                const int64_t n_keys = units[id].n_keys;
                 int64_t k0 = 0;
                 int c = 0;
-                while (left > 0) {
+                while (k0 < n_keys) {
+                    const int pth = cta < started ? 0 : path;
+                    const PathCost& pc = cost[pth];
+                    const bool narrow = pth == 0;          // only narrow units are line-filled on the tensor path
+                    const int64_t tns = narrow ? narrow_tile_ns : tns_of[(size_t)id];
+                    const int64_t item_ns = narrow ? narrow_item_ns : pc.item_ns;
+                    const int64_t left = (n_keys - k0 + pc.gran - 1) / pc.gran;
                     const bool last_cta = cta + 1 >= n_ctas;
-                    const int64_t start = pc.item_ns + (has_phase ? 0 : pc.phase_ns);
+                    const int64_t start = item_ns + ((has_phase || cta < started) ? 0 : pc.phase_ns);
                     const int64_t room = cap - load[(size_t)cta] - start;
                     int64_t take;
                     if (last_cta) {
                         take = left;
-                        if (load[(size_t)cta] + start + take * pc.tile_ns > cap) fits = false;
-                    } else if (left * pc.tile_ns <= room + pc.item_ns / 2) {
+                        if (load[(size_t)cta] + start + take * tns > cap) fits = false;
+                    } else if (left * tns <= room + item_ns / 2) {
                         take = left;                     // finishing here is cheaper than another item elsewhere
-                    } else if (room < pc.tile_ns * 2) {
-                        next_cta();                      // not worth starting an item for so little
+                    } else if (room < tns * 2) {
+                        ++cta;                           // not worth starting an item for so little
+                        has_phase = false;
                         continue;
                     } else {
-                        take = std::max<int64_t>(1, room / pc.tile_ns);
+                        take = std::max<int64_t>(1, room / tns);
                     }
-                    const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
-                    if (emit) out[1].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
+                    const int64_t k1 = std::min<int64_t>(n_keys, k0 + take * pc.gran);
+                    if (emit) out[pth].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
                     else if (!fits) return false;
-                    load[(size_t)cta] += start + take * pc.tile_ns;
+                    load[(size_t)cta] += start + take * tns;
                     has_phase = true;
-                    left -= take;
                     k0 = k1;
                     ++c;
-                    if (!last_cta && left > 0) next_cta();
+                    if (!last_cta && k0 < n_keys) { ++cta; has_phase = false; }
                 }
             }
-        }
+            return true;
+        };
+        // narrow tensor units: on the span CTAs first, then on fresh CTAs (which pay the phase start)
+        if (!line_fill(0, tensor_narrow, used)) return false;
+        if (!line_fill(1, *ids[1], ids[1]->empty() ? 0 : used)) return false;
+        std::stable_sort(out[0].begin(), out[0].end(), [](const Piece& x, const Piece& y) { return x.cta < y.cta; });
         return fits;
     };
     // Smallest limit that fits, by bisection (the loads are monotone in the limit up to rounding).
     // The probes only ask whether a limit fits; the pieces are built once, for the limit found.
-    int64_t lo = std::max<int64_t>(1, total / n_ctas);
+    int64_t lo = std::max<int64_t>(1, total / n_ctas * 3 / 4);     // (decode rows on span CTAs cost less than assumed in `total`)
     int64_t hi = lo + lo / 4 + kTensorCost.item_ns + kTensorCost.phase_ns + kCudaCost.phase_ns;
     while (!fill(hi, best, false)) { lo = hi; hi += hi / 2; }
     for (int iter = 0; iter < 24 && hi - lo > std::max<int64_t>(50, hi / 128); ++iter) {      // to 0.8 %

@@ -68,6 +68,22 @@ def test_eight_heads_per_kv_head_decode_rows_take_the_tensor_path():
     assert 0 < plan.info["num_items_tensor"] < plan.info["num_items"]
 
 
+def test_decode_rows_on_span_ctas_run_as_narrow_tensor_items():
+    """Default policy, 4 heads per kv head: CTAs that hold span units take decode rows as tensor-core
+    items of 4 rows (cut where the CTA is full), the other CTAs run them on the CUDA-core body."""
+    shape = W.Shape(8, 2, 128, 16)
+    ctx = [1900, 40, 2500, 3, 700, 1200, 0, 333] + [900 + 37 * i for i in range(24)]
+    ql = [40, 1, 1, 9, 1, 64, 1, 1] + [1] * 24
+    wl = W.make_single_step("hybrid", shape, ctx, ql, seed=83)
+    _, _, plan = run_and_check(wl, what="decode rows beside spans", num_sms=12)
+    items = plan.items()
+    tens, cuda = items[items["path"] == 1], items[items["path"] == 0]
+    assert ((tens["ntok"] == 1).sum() > 0) and len(cuda) > 0
+    assert not set(tens["cta"].tolist()) & set(cuda["cta"].tolist())
+    out_a, lse_a, _ = run_and_check(wl, what="all rows on the CUDA-core body", flags=B.PLAN_NO_TENSOR_PATH)
+    out_b, lse_b, _ = run_and_check(wl, what="all rows on the tensor-core body", tensor_min_rows=1)
+
+
 def test_results_are_bitwise_reproducible():
     wl = W.make_config(1)
     a = gpu_step(wl, wl.steps[0])

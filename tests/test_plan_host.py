@@ -179,11 +179,18 @@ def test_mixed_batch_spans_stay_whole_and_loads_balance():
     span = items[items["path"] == 1]
     dec = items[items["path"] == 0]
     assert len(span) and len(dec)
-    assert (span["kv0"] % 128 == 0).all() and (dec["kv0"] % 96 == 0).all()
+    assert (span["kv0"] % 128 == 0).all() and (dec["kv0"] % 16 == 0).all()
+    # a CTA runs one body only: where span units sit, decode rows ride along as narrow tensor-core items
+    assert not set(span["cta"].tolist()) & set(dec["cta"].tolist())
+    narrow = span[span["ntok"] * 4 < 32]
+    assert len(narrow) and (narrow["ntok"] == 1).all()
+    wide_ctas = set(span[span["ntok"] * 4 >= 32]["cta"].tolist())
+    assert set(narrow["cta"].tolist()) <= wide_ctas
     # a span unit covers up to 256 (token, head) rows: 64 tokens at 4 heads per kv head
     assert span["ntok"].max() <= 64 and (span["tok0"] % 64 == 0).all()
-    units = {(int(it["seq"]), int(it["kv_head"]), int(it["tok0"])) for it in span}
-    pieces = len(span) / len(units)
+    wide = span[span["ntok"] * 4 >= 32]
+    units = {(int(it["seq"]), int(it["kv_head"]), int(it["tok0"])) for it in wide}
+    pieces = len(wide) / len(units)
     assert pieces < 1.6, pieces          # most span units are one item (no partial rows, no merge)
     # modelled load per CTA in KV tiles (a span tile of two row tiles counts double)
     load = np.zeros(148)
