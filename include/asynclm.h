@@ -74,9 +74,11 @@ typedef struct asynclm_plan_options {
                                  the work items roughly fill the machine; a value >= the longest
                                  context disables splitting */
     int32_t tensor_min_rows;  /* new tokens of a sequence use the tensor-core path when
-                                 G * q_len >= this; 0 = default: 32 (decode rows stay on the
-                                 CUDA-core path) for G <= 4, and 8 for G = 8, where the CUDA-core
-                                 path is bound by its arithmetic rather than by memory;
+                                 G * q_len >= this; 0 = default: 32 for G <= 4 (a decode row
+                                 then runs on the CUDA-core path, except on a CTA that also
+                                 holds span tiles, where it runs as a narrow tensor-core item),
+                                 and 8 for G = 8, where the CUDA-core path is bound by its
+                                 arithmetic rather than by memory;
                                  INT32_MAX keeps every row on the CUDA-core path, like
                                  ASYNCLM_PLAN_NO_TENSOR_PATH */
     int32_t flags;            /* ASYNCLM_PLAN_* */
@@ -153,7 +155,8 @@ int asynclm_plan_workspace_size(const asynclm_shape* shape, const asynclm_plan_o
  * (long contexts are split; partial results are merged by log-sum-exp inside asynclm_attn_mixed),
  * assigns the items to persistent CTAs under the smallest per-CTA load limit that fits (span tiles
  * are kept whole where possible, largest first; decode rows fill the CTAs up and are cut only
- * where a CTA is full), then enqueues ONE host->device copy of the packed plan on `stream`.
+ * where a CTA is full; a CTA runs one kernel body only, so decode rows placed beside span tiles
+ * become tensor-core items), then enqueues ONE host->device copy of the packed plan on `stream`.
  *
  *   host_ws / host_bytes  host memory (8-byte aligned; pinned recommended) that must stay untouched
  *                         until the copy has completed and for as long as the plan is used.
