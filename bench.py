@@ -33,7 +33,7 @@ WORKLOAD = "config2-llama3-8b-mixed-batch"       # the configuration the metric 
 WORKLOADS = {2: WORKLOAD, 3: "config3-large-batch-gqa8", 4: "config4-long-context-split-kv"}
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on this workload
 # (profiles/attn_fused_kernel_config2.md); None whenever the kernel has changed since that capture
-TRAFFIC_BYTES_PER_LAUNCH = 328_686_592
+TRAFFIC_BYTES_PER_LAUNCH = 327_827_712
 
 
 def measured_peaks():
