@@ -200,6 +200,32 @@ def test_mixed_batch_spans_stay_whole_and_loads_balance():
     assert p.info["launches_attn"] == 2 and p.info["num_split_units"] > 0
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_random_mixed_batches_are_covered_once_under_the_default_policy(seed):
+    """Spans, decode rows, paused and empty-context sequences at head_dim 128 (both kernel bodies in
+    play): every (sequence, kv head, token, key) is covered by exactly one item, whatever the SM count."""
+    g = np.random.default_rng(100 + seed)
+    n = int(g.integers(3, 40))
+    ctx = g.integers(0, 3000, n)
+    ctx[g.random(n) < 0.15] = 0
+    ql = np.ones(n, dtype=np.int64)
+    spans = g.random(n) < 0.3
+    ql[spans] = g.integers(2, 80, int(spans.sum()))
+    ql[g.random(n) < 0.1] = 0
+    ql[(ctx == 0) & (ql == 0)] = 1
+    heads = [(8, 2), (4, 1), (16, 2), (4, 4)][seed % 4]
+    shape = W.Shape(heads[0], heads[1], 128, 16)
+    wl = W.make_single_step("rnd", shape, ctx.tolist(), ql.tolist(), seed=seed)
+    for sms in (3, 20, 148):
+        p = plan(wl, num_sms=sms)
+        items = check_cover(wl, p)
+        assert items["cta"].max() < sms
+        t, c = items[items["path"] == 1], items[items["path"] == 0]
+        group = heads[0] // heads[1]
+        if group <= 4 and len(t) and len(c):
+            assert not set(t["cta"].tolist()) & set(c["cta"].tolist())
+
+
 def test_decode_only_batch_has_no_span_items():
     ctx, ql, num_pages, q_indptr, page_indptr, page_indices = _llama_lengths(1)
     ql[:] = 1
