@@ -238,10 +238,11 @@ constexpr int kWholeUnitMinRows = 32;
 // Decode units that a span CTA takes along on the tensor-core body at most (estimated from its room).
 constexpr int64_t kMaxNarrowUnitsPerCta = 4;
 
-// Default policy for the fused kernel, in which every persistent CTA runs its tensor-core items and
-// then its CUDA-core items: units are weighted with the measured costs and dealt under a per-CTA load
-// limit (see `fill` below); the smallest limit that fits is found by bisection, so that all CTAs
-// finish together as far as the cost model holds.
+// Default policy for the fused kernel, in which a persistent CTA runs its tensor-core items and then,
+// if it has any, its CUDA-core items: units are weighted with the measured costs and dealt under a
+// per-CTA load limit (see `fill` below), where decode rows placed on a CTA with span work normally
+// become tensor-core items so that the CTA runs one body only; the smallest limit that fits is found
+// by bisection, so that all CTAs finish together as far as the cost model holds.
 void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& ids_cuda,
                   std::vector<UnitBuild>& units, int group, int n_ctas, std::vector<Item>& items,
                   std::vector<int32_t>& cta_indptr_cuda, std::vector<int32_t>& cta_indptr_tensor,
