@@ -234,14 +234,8 @@ __device__ __forceinline__ TItem load_titem(const Work* rec, bool valid) {
     return r;
 }
 
-// Register shares of the fused kernel's tensor-core phase (512 threads launched with 128 each):
-// softmax warps 0-7, the producer/MMA warpgroup 8-11, and warps 12-15, which idle in this phase.
-constexpr int kRegsSoftmaxFused = 168, kRegsIssueFused = 80, kRegsIdleFused = 24;
-static_assert(256 * kRegsSoftmaxFused + 128 * kRegsIssueFused + 128 * kRegsIdleFused <= 65536, "register split");
-
-// The whole kernel body.  FUSED: called by all 16 warps of the fused kernel (warps 12-15 only take
-// part in the CTA-wide barriers), with `smem` 1024-byte aligned.
-template <int G, bool FUSED>
+// The whole kernel body, called by all twelve warps with `smem` 1024-byte aligned.
+template <int G>
 __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
                                         const __nv_bfloat16* __restrict__ pool,
                                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
@@ -286,10 +280,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
     tc_fence_after();
     const uint32_t tmem = *tmem_ptr;
 
-    if (warp >= 12) {
-        if constexpr (FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIdleFused));
-    } else if (warp >= 8) {
-      if constexpr (FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsIssueFused));
+    if (warp >= 8) {
       if (warp == kProducerWarpK || warp == kProducerWarpV) {
         // ------------------------------------------------------------------ producer warps
         const int which = warp == kProducerWarpV ? 1 : 0;       // 0: K tiles, 1: V tiles
@@ -443,7 +434,6 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         __syncwarp();
       }
     } else {
-        if constexpr (FUSED) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxFused));
         // ------------------------------------------------------------------ softmax / epilogue groups
         const int b = warp >> 2;                   // softmax group
         const int m = threadIdx.x & 127;           // row of the group's tile = tensor-memory lane

@@ -1,20 +1,28 @@
-// CUDA-core attention for decode rows (and spans too short for the tensor-core path).
+// Warp-level attention for decode rows (and spans too short for the tcgen05 path).
 //
 // Each new token attends to its sequence's whole cached context plus its own span up to itself
 // (paper Section 3.2 / 5.3: interrupt tokens are appended to the context and processed in the next
-// decoding step, next to the other sequences' one-token decodes).  This path is bound by HBM
-// bandwidth: every K/V row is read once and used by the G query heads that share the kv head.
+// decoding step, next to the other sequences' one-token decodes).  This path has to be bound by HBM
+// bandwidth: every K/V row is read once and used by the G query heads that share the kv head, i.e.
+// G multiply-adds per byte, far below the machine's ridge.  Doing those multiply-adds on the fp32
+// pipes costs an unpack and two FMAs per bf16 pair and made the path instruction-bound, so the two
+// small contractions of a page run on warp-level tensor instructions (mma.sync m16n8k16) with the
+// KEYS on the M axis, which wastes nothing on padding query rows:
+//     S^T [16 keys x 8 columns]   = K_page [16 x d]      . Q^T [d x 8]        (d / 16 instructions)
+//     O^T [d x 8 columns]        += V_page^T [d x 16]    . P^T [16 x 8]       (d / 16 instructions)
+// A column is one (token, head) pair of the unit: up to 8 / G consecutive tokens times the G heads
+// of the kv head; unused columns carry zeros.  About 70 warp instructions per page instead of 700.
 //
 // Structure: one persistent CTA per SM walks the item list the planner gave it.  A producer warp
-// streams the items' K/V pages (contiguous 16-token blocks) into a shared-memory ring with bulk
-// asynchronous copies that complete on mbarriers, together with a small descriptor and the query
-// rows of each item.  Twelve consumer warps each take 8 rows of a 96-row tile: fp32 dot products
-// with packed two-wide FMAs, a select-free transposing shuffle reduction, softmax against a lazily
-// updated reference maximum, and the P.V update; at the end of an item the warps' states are merged
-// through shared memory and written either as final bf16 output or as an fp32 partial for the
-// split-KV merge.  The path is bound by instruction latency rather than by any one pipe, so the
-// warp count matters: registers are moved from the producer's warpgroup to the consumers
-// (setmaxnreg) to keep twelve of them resident.
+// streams the items' pages into a shared-memory ring of 128-key stages, one tiled TMA copy per
+// (page, kv head) that brings the K block and the V block together and lands them with the
+// 128-byte swizzle that makes ldmatrix conflict-free; a small descriptor and the unit's query rows
+// travel with each stage.  Eight consumer warps take one page of a stage each: ldmatrix, the two
+// contractions, softmax against a lazily moved reference maximum on the accumulator fragment
+// (4 values per thread), P transposed in registers (movmatrix) into the B operand.  At the end of
+// an item the warps' states are merged through the shared memory of the item's last stage (which
+// is idle by then) and written either as final bf16 output or as an fp32 partial for the split-KV
+// merge.
 //
 // Every wait is bounded: a wait that runs out sets the plan's device status word and a CTA-wide
 // abort flag, after which all loops fall through and the kernel returns.
@@ -28,29 +36,25 @@ namespace asynclm {
 
 namespace dec {
 
-constexpr int kWarps = 12;                   // consumer warps (three warpgroups)
-constexpr int kThreads = (kWarps + 4) * 32;  // + the producer's warpgroup (one working warp)
-constexpr int kRowsPerWarp = 8;
-// A warp works on at most 4 query heads (the accumulators of more do not fit its registers).  With
-// 8 heads per kv head the warps split into two halves that take 4 heads each and share the K/V
-// rows in shared memory: 6 row blocks x 2 head halves, 48-row tiles instead of 96.
-__host__ __device__ constexpr int head_splits(int group) { return group > 4 ? group / 4 : 1; }
-// Register budget: the CTA is launched with 512 x 128 registers; the producer's warpgroup gives
-// most of its share back and the consumers take it: 384 x 160 + 128 x 24 = 64512 <= 65536.
-constexpr int kRegsConsumer = 152, kRegsProducer = 56;
-static_assert(kWarps * 32 * kRegsConsumer + 128 * kRegsProducer <= 65536, "register split");
-constexpr float kRescaleThreshold = 16.f;    // log2 units a score may exceed the reference max by
+constexpr int kWarps = 8;                    // consumer warps: one page of a 128-key stage each
+constexpr int kProducerWarp = kWarps;        // the warp behind them streams the pages
+constexpr int kThreads = (kWarps + 2) * 32;  // standalone kernel: consumers, producer, one spare warp
+constexpr int kCols = 8;                     // (token, head) columns of a unit: the N of the MMAs
+constexpr int kTileTok = kWarps * kPage;     // keys per ring stage
+constexpr float kRescaleThreshold = 8.f;     // log2 units a score may exceed the reference max by
 constexpr long long kWaitCycles = 2000000000ll;
 
 constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
 
 struct TileDesc {
     int32_t flags;
-    int32_t rows;         // valid rows in this tile
-    int32_t out_row;      // global token row of the item
+    int32_t rows;         // keys of this stage that some column may see
+    int32_t lim0;         // keys of this stage that column 0's token sees (may be <= 0 or > rows)
+    int32_t ntok;         // tokens of the unit
+    int32_t out_row;      // global token row of the unit's first token
     int32_t kv_head;
     int32_t partial_row;  // -1: final output
-    int32_t pad[3];
+    int32_t pad;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -98,99 +102,84 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 
-// One tiled TMA copy fetches the K block and the V block of a (page, kv head): the pool is described
-// to the TMA unit as a 5-D tensor [pages][2][Hkv][16][d] and the box spans (d, 16, 1, 2, 1), i.e. two
-// separate 16 x d blocks of global memory that land back to back in shared memory.  (A bulk/TMA
-// copy costs about 70 cycles plus 1 cycle per 107 bytes on this part, so halving the number of
-// copies matters.)  No multicast.
+// One tiled TMA copy fetches the K block and the V block of a (page, kv head).  The pool is
+// described to the TMA unit as a 5-D tensor
+//     (64 values, 16 slots, d / 64 halves of a row, Hkv heads, 2 * pages [page * 2 + K|V])
+// and the box spans (64, 16, d / 64, 1, 2): two separate 16 x d blocks of global memory that land
+// back to back in shared memory as [K|V][half][slot][64 values], every 128-byte row swizzled by its
+// slot (16-byte piece c of slot s sits at piece c ^ (s & 7)).  No multicast.
 __device__ __forceinline__ void tma_page_kv(uint32_t dst, const CUtensorMap* map, int kv_head, int page, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-        ::"r"(dst), "l"(map), "r"(0), "r"(0), "r"(kv_head), "r"(0), "r"(page), "r"(bar) : "memory");
+        ::"r"(dst), "l"(map), "r"(0), "r"(0), "r"(0), "r"(kv_head), "r"(2 * page), "r"(bar) : "memory");
 }
 
-__device__ __forceinline__ float2 unpack2(uint32_t w) { return make_float2(bf16_lo(w), bf16_hi(w)); }
-
-// Transposing reduction over the LPR lanes that share a row.  Every lane starts with N values that
-// must each be summed over the LPR lanes; each stage halves the number of values a lane keeps
-// (while more than one is left) and adds the partner's copy of the kept half.  No selects are
-// needed because a lane fills its slots in a lane-dependent order: slot k of lane `sub` holds the
-// value with true index k ^ mask(sub), mask(sub) = sub * N / LPR (or sub >> log2(LPR / N) when
-// N < LPR), so at every stage all lanes keep the lower half of their slots and send the upper
-// half.  Afterwards slot f of lane `sub` holds the complete sum of true index
-// sub * (N / LPR) + f (or sub >> log2(LPR / N) when N < LPR, duplicated over neighbouring lanes).
-template <int N, int OFF, int NMAX>
-__device__ __forceinline__ void transpose_reduce(float (&v)[NMAX]) {
-    if constexpr (OFF >= 1) {
-        if constexpr (N > 1) {
-#pragma unroll
-            for (int j = 0; j < N / 2; ++j)
-                v[j] += __shfl_xor_sync(0xffffffffu, v[j + N / 2], OFF);
-            transpose_reduce<N / 2, OFF / 2, NMAX>(v);
-        } else {
-            v[0] += __shfl_xor_sync(0xffffffffu, v[0], OFF);
-            transpose_reduce<1, OFF / 2, NMAX>(v);
-        }
-    }
+// Four 8x8 b16 matrices; lane l gives the address of row l % 8 of matrix l / 8; thread (g, t) =
+// (lane / 4, lane % 4) receives elements [g][2t], [g][2t+1] of each (transposed: [2t][g], [2t+1][g]).
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// Transpose of an 8x8 b16 matrix held one row per four threads.
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+// D (16x8, fp32) += A (16x16, bf16, row) . B (16x8, bf16, col).  Thread (g, t) holds
+//   A: [g][2t..], [g+8][2t..], [g][2t+8..], [g+8][2t+8..]   B: [2t..][g], [2t+8..][g]
+//   D: [g][2t], [g][2t+1], [g+8][2t], [g+8][2t+1]
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-constexpr int ilog2(int x) { return x <= 1 ? 0 : 1 + ilog2(x / 2); }
-
-template <int D, int G, int HS = 1>     // G: heads per warp, HS: head halves per CTA
+template <int D>
 struct Geometry {
-    static constexpr int LPR = D / 8;                 // lanes per row (16 bytes each)
-    static constexpr int TPW = 32 / LPR;              // rows per warp-wide shared-memory load
-    static constexpr int NR = kRowsPerWarp / TPW;     // rows per lane
-    static constexpr int NV = NR * G;                 // partial dot products per lane
-    static constexpr int NF = NV >= LPR ? NV / LPR : 1;              // finished scores per lane
-    static constexpr int DUP_SHIFT = NV >= LPR ? 0 : ilog2(LPR / NV); // lanes holding duplicates
-    static constexpr int PAGE_BYTES = kPage * D * 2;
-    static constexpr int ROW_BLOCKS = kWarps / HS;
-    static constexpr int TILE_TOK = ROW_BLOCKS * kRowsPerWarp;          // rows per ring stage: 96 or 48
-    // a stage holds, page after page, the page's K block followed by its V block
-    static constexpr int STAGE_BYTES = (TILE_TOK / kPage) * 2 * PAGE_BYTES;
-    static constexpr int Q_BYTES = G * HS * D * 2;
-    static constexpr int STAT_FLOATS = (kWarps * G + 7) / 8 * 8;         // max (or sum) array, padded to 32 bytes
-    static constexpr int MERGE_FLOATS = 2 * STAT_FLOATS + kWarps * G * D;  // one merge buffer
-    // A lane's slot (i, g) holds the partial score of true row i ^ xi and true head g ^ xg, with
-    // (xi, xg) = (mask / G, mask % G) and mask as in transpose_reduce.  The finished score of a
-    // lane's slot (i, g) sits in slot score_slot(i, g) of the lane whose index differs from its own
-    // by score_xor(i, g).
-    __host__ __device__ static constexpr int score_xor(int i, int g) {
-        return NV >= LPR ? (i * G + g) / NF : (i * G + g) << DUP_SHIFT;
-    }
-    __host__ __device__ static constexpr int score_slot(int i, int g) { return NV >= LPR ? (i * G + g) % NF : 0; }
+    static constexpr int HALVES = D / 64;                       // 128-byte pieces of a K or V row
+    static constexpr int BLOCK_BYTES = kPage * D * 2;           // one (page, K|V, head) block
+    static constexpr int PAGE_BYTES = 2 * BLOCK_BYTES;          // K block + V block: one TMA copy
+    static constexpr int STAGE_BYTES = kWarps * PAGE_BYTES;     // 64 KiB at d = 128
+    static constexpr int Q_BYTES = kCols * D * 2;               // the unit's query rows, [column][d]
+    static constexpr int KSTEPS = D / 16;
+    // merge area of a warp inside its page slot: O^T as [column][d + 4] fp32 (the pad keeps the
+    // fragment stores conflict-free), then the columns' reference maxima and sums
+    static constexpr int O_STRIDE = D + 4;
+    static constexpr int STATE_FLOATS = kCols * O_STRIDE + 2 * kCols;
+    static_assert(STATE_FLOATS * 4 <= PAGE_BYTES, "a warp's merge state must fit its page slot");
 };
 
-template <int D, int GT>
+template <int D>
 size_t smem_bytes(int stages) {
-    using Geo = Geometry<D, GT / head_splits(GT), head_splits(GT)>;
-    return (size_t)stages * (Geo::STAGE_BYTES + Geo::Q_BYTES + sizeof(TileDesc) + 16) +
-           2 * Geo::MERGE_FLOATS * sizeof(float) + 3 * 8 + 16 + 1024;
+    using Geo = Geometry<D>;
+    return (size_t)stages * (Geo::STAGE_BYTES + Geo::Q_BYTES + sizeof(TileDesc) + 16) + 8 + 16 + 1024;
 }
 
-// The whole kernel body.  FUSED: the CTA has just finished the tensor-core phase of the fused
-// kernel, in which warps 0-7 held 168 registers, warps 8-11 held 80 and warps 12-15 held 24.
-template <int D, int GT, bool FUSED>
+// The whole kernel body: warps 0-7 consume, warp 8 produces, any further warps of the CTA return at
+// once (the fused kernel has twelve).
+template <int D, int GT>
 __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap* kv_map,
                                             const __nv_bfloat16* __restrict__ q,
                                             __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                                             int S, uint8_t* smem) {
-    constexpr int HS = head_splits(GT);     // head halves
-    constexpr int G = GT / HS;              // query heads per warp
-    using Geo = Geometry<D, G, HS>;
-    constexpr int LPR = Geo::LPR, TPW = Geo::TPW, NR = Geo::NR, NV = Geo::NV, NF = Geo::NF;
-    constexpr int RB = Geo::ROW_BLOCKS, kTileTok = Geo::TILE_TOK;
-    uint8_t* stage_base = smem;
+    using Geo = Geometry<D>;
+    constexpr int G = GT;
+    static_assert(G <= kCols && kCols % G == 0, "heads per kv head must divide the column count");
+    uint8_t* stage_base = smem;                                        // 1024-byte aligned
     uint8_t* q_base = stage_base + (size_t)S * Geo::STAGE_BYTES;
-    float* merge_base = (float*)(q_base + (size_t)S * Geo::Q_BYTES);
-    TileDesc* desc = (TileDesc*)(merge_base + 2 * Geo::MERGE_FLOATS);
-    uint64_t* bars = (uint64_t*)(desc + S);      // full[S], empty[S], merge[2]
-    volatile int* abort_flag = (volatile int*)(bars + 2 * S + 2);
+    TileDesc* desc = (TileDesc*)(q_base + (size_t)S * Geo::Q_BYTES);
+    uint64_t* bars = (uint64_t*)(desc + S);      // full[S], empty[S], merge
+    volatile int* abort_flag = (volatile int*)(bars + 2 * S + 1);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), mbar0 = smem_u32(bars + 2 * S);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), mbar = smem_u32(bars + 2 * S);
 
     if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(kv_map));
     if (threadIdx.x == 0) {
@@ -198,8 +187,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, kWarps);
         }
-        mbar_init(mbar0, kWarps);
-        mbar_init(mbar0 + 8, kWarps);
+        mbar_init(mbar, kWarps);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -209,26 +197,24 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
     const int Hq = p.num_q_heads;
 
     if (warp >= kWarps) {
-        if constexpr (!FUSED) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsProducer));
-        else asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsProducer));      // idled with 24 so far
-        if (warp > kWarps) return;      // the other warps of the producer's warpgroup have nothing to do
+        if (warp != kProducerWarp) return;      // spare warps have nothing to do
         // ------------------------------------------------------------------ producer warp
-        // The page ids of the next 32 pages (8 tiles) and the descriptors of the next two items are
-        // fetched ahead of use, so that no global-load latency sits between two tiles.
-        struct PItem { int kv0, kv_end, q_row0, kv_head, partial_row, page0; };
+        // The page ids of the next 32 pages (4 stages) and the descriptors of the next two items are
+        // fetched ahead of use, so that no global-load latency sits between two stages.
+        struct PItem { int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row, page0; };
         int n = 0;
         // the CTA's header gives its item range, its first item and that item's first 32 page ids in
         // one round trip to memory
         const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
         const int i0 = head[2], i1 = head[3];
         auto load_item = [&](int ii) {
-            PItem r{0, 0, 0, 0, -1, 0};
+            PItem r{0, 0, 0, 0, 0, 0, -1, 0};
             if (ii < i1) {
                 const int4* src = ii == i0 ? reinterpret_cast<const int4*>(head + kHeadWorkCuda)
                                            : reinterpret_cast<const int4*>(p.works + ii);
                 const int4 a = __ldg(src), b = __ldg(src + 1);
-                r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z;
-                r.kv_head = b.y; r.partial_row = b.z; r.page0 = b.w;
+                r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z; r.ntok = a.w;
+                r.kv_limit0 = b.x; r.kv_head = b.y; r.partial_row = b.z; r.page0 = b.w;
             }
             return r;
         };
@@ -237,8 +223,8 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             const int idx = first_page + lane;
             return idx < npg ? __ldg(p.page_indices + it.page0 + idx) : 0;
         };
-        constexpr int kPagesPerTile = kTileTok / kPage;
-        constexpr int kGroupTiles = 32 / kPagesPerTile;
+        constexpr int kPagesPerTile = kTileTok / kPage;       // 8
+        constexpr int kGroupTiles = 32 / kPagesPerTile;       // 4
         bool ok = true;
         PItem cur = load_item(i0), nxt = load_item(i0 + 1);
         int pages_cur = head[kHeadPagesCuda + lane];
@@ -264,25 +250,31 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                         TileDesc d;
                         d.flags = (first ? kFlagFirst : 0) | (t == ntiles - 1 ? kFlagLast : 0);
                         d.rows = rows;
+                        d.lim0 = cur.kv_limit0 - base;
+                        d.ntok = cur.ntok;
                         d.out_row = cur.q_row0;
                         d.kv_head = cur.kv_head;
                         d.partial_row = cur.partial_row;
+                        d.pad = 0;
                         desc[s] = d;
                         mbar_arrive_expect_tx(full0 + 8 * s,
-                                              (uint32_t)(npages * 2 * Geo::PAGE_BYTES + (first ? Geo::Q_BYTES : 0)));
+                                              (uint32_t)(npages * Geo::PAGE_BYTES + (first ? cur.ntok * G * D * 2 : 0)));
                     }
                     __syncwarp();
-                    const int64_t page = __shfl_sync(0xffffffffu, pages_cur,
-                                                     (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
+                    const int page = __shfl_sync(0xffffffffu, pages_cur,
+                                                 (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
                     if (lane < npages)
-                        tma_page_kv(smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + lane * 2 * Geo::PAGE_BYTES),
-                                    kv_map, cur.kv_head, (int)page, full0 + 8 * s);
-                    if (first && lane == 31) {
-                        const __nv_bfloat16* src = q + ((size_t)cur.q_row0 * Hq + (size_t)cur.kv_head * GT) * D;
-                        bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES), src, Geo::Q_BYTES, full0 + 8 * s);
+                        tma_page_kv(smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + (size_t)lane * Geo::PAGE_BYTES),
+                                    kv_map, cur.kv_head, page, full0 + 8 * s);
+                    // the unit's query rows: G * d contiguous values per token, columns in (token, head) order
+                    if (first && lane >= 16 && lane - 16 < cur.ntok) {
+                        const int tok = lane - 16;
+                        const __nv_bfloat16* src = q + ((size_t)(cur.q_row0 + tok) * Hq + (size_t)cur.kv_head * G) * D;
+                        bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES + (size_t)tok * G * D * 2), src,
+                                 G * D * 2, full0 + 8 * s);
                     }
-                    // page ids of the next group of tiles (or of the next item), requested only after this
-                    // group's first tile is on its way: the next item's descriptor may still be in flight
+                    // page ids of the next group of stages (or of the next item), requested only after this
+                    // group's first stage is on its way: the next item's descriptor may still be in flight
                     if (t == t0) {
                         if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
                         else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
@@ -314,26 +306,21 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
 
     // ---------------------------------------------------------------------- consumer warps
     pdl_wait();      // outputs may be written only after the kernel in front has completed
-    if constexpr (FUSED) {
-        if (warp < 8) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
-        else asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
-    } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsConsumer));
-    }
-    const int sub = lane % LPR;
-    const int grp = lane / LPR;
-    const int my_row = (sub >> 2) * TPW + grp;   // row (within the warp's 8) of this lane's scores
-    const int mask = NV >= LPR ? sub * NF : sub >> Geo::DUP_SHIFT;
-    const int xi = mask / G;                     // this lane's slot i holds true row i ^ xi
-    const int xg = mask % G;                     // and its slot g holds true head g ^ xg
+    const int g = lane >> 2, t4 = lane & 3;      // fragment coordinates
     const float qscale = p.sm_scale * kLog2e;
+    // ldmatrix row addresses inside a page slot, without the per-step piece index:
+    //   K (plain): matrices (keys 0-7, k 0-7), (keys 8-15, k 0-7), (keys 0-7, k 8-15), (keys 8-15, k 8-15)
+    //   V (transposed): (keys 0-7, d 0-7), (keys 0-7, d 8-15), (keys 8-15, d 0-7), (keys 8-15, d 8-15)
+    const int k_key = (lane & 7) + ((lane >> 3) & 1) * 8, k_piece = lane >> 4;
+    const int v_key = (lane & 7) + (lane >> 4) * 8, v_piece = (lane >> 3) & 1;
+    const uint32_t k_row = (uint32_t)k_key * 128u, v_row = (uint32_t)Geo::BLOCK_BYTES + (uint32_t)v_key * 128u;
+    const uint32_t k_swz = (uint32_t)(k_key & 7), v_swz = (uint32_t)(v_key & 7);
 
-    float2 q2[G][4];
-    float2 o2[G][4];
-    float m_ref[G];
-    float m_own[NF], l_own[NF];
+    uint32_t qb[Geo::KSTEPS][2];      // B fragments of Q^T: column g, values 16 ks + 2 t4 (+1) and + 8
+    float o[Geo::KSTEPS][4];          // O^T: rows d = 16 i + g (+8), columns 2 t4, 2 t4 + 1
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;      // of columns 2 t4 and 2 t4 + 1
+    int32_t cur_out_row = 0, cur_kv_head = 0, cur_partial = -1, cur_ntok = 1;
     int item_count = 0;
-    int32_t cur_out_row = 0, cur_kv_head = 0, cur_partial = -1;
 
     for (int n = 0;; ++n) {
         const int s = n % S;
@@ -341,197 +328,164 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status, 2)) break;
         const TileDesc d = desc[s];
         if (d.flags & kFlagEnd) break;
+        uint8_t* stage = stage_base + (size_t)s * Geo::STAGE_BYTES;
         if (d.flags & kFlagFirst) {
             const uint8_t* qs = q_base + (size_t)s * Geo::Q_BYTES;
+            const bool col_valid = g < d.ntok * G;
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const uint4 w = *reinterpret_cast<const uint4*>(qs + ((size_t)((warp / RB) * G + (g ^ xg)) * D + sub * 8) * 2);
-                q2[g][0] = unpack2(w.x); q2[g][1] = unpack2(w.y);
-                q2[g][2] = unpack2(w.z); q2[g][3] = unpack2(w.w);
+            for (int ks = 0; ks < Geo::KSTEPS; ++ks) {
+                const uint32_t* src = reinterpret_cast<const uint32_t*>(qs + ((size_t)g * D + ks * 16 + t4 * 2) * 2);
+                qb[ks][0] = col_valid ? src[0] : 0u;
+                qb[ks][1] = col_valid ? src[4] : 0u;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    q2[g][j].x *= qscale; q2[g][j].y *= qscale;
-                    o2[g][j] = make_float2(0.f, 0.f);
-                }
-                m_ref[g] = -INFINITY;
+                for (int e = 0; e < 4; ++e) o[ks][e] = 0.f;
             }
-#pragma unroll
-            for (int f = 0; f < NF; ++f) { m_own[f] = -INFINITY; l_own[f] = 0.f; }
-            cur_out_row = d.out_row; cur_kv_head = d.kv_head; cur_partial = d.partial_row;
+            m0 = m1 = -INFINITY;
+            l0 = l1 = 0.f;
+            cur_out_row = d.out_row; cur_kv_head = d.kv_head; cur_partial = d.partial_row; cur_ntok = d.ntok;
         }
-        const int rows = d.rows;
-        const int blk = warp % RB;      // row block of the tile; warp / RB is the head half
-        const bool active = blk * kRowsPerWarp < rows;
-        uint4 kw[NR], vw[NR];
-        if (active) {
-            // the warp's 8 rows are one half of a page: [page][K 16 rows | V 16 rows]
-            const uint8_t* ks = stage_base + (size_t)s * Geo::STAGE_BYTES + (size_t)(blk >> 1) * 2 * Geo::PAGE_BYTES +
-                                (size_t)((blk & 1) * kRowsPerWarp) * (D * 2) + lane * 16;
+        const int key0 = warp * kPage;                    // this warp's page inside the stage
+        if (key0 < d.rows) {
+            const uint32_t page_smem = smem_u32(stage) + (uint32_t)warp * Geo::PAGE_BYTES;
+            const int valid = d.rows - key0;              // slots of the page that hold keys of the sequence
+            if (valid < kPage) {
+                // Slots past the sequence's end hold whatever was in the page before: their scores are
+                // masked below, but 0 * NaN would still poison P V, so their V rows are cleared.
+                for (int r = valid + (lane >> 4); r < kPage; r += 2)
 #pragma unroll
-            for (int i = 0; i < NR; ++i) {
-                kw[i] = *reinterpret_cast<const uint4*>(ks + (size_t)(i ^ xi) * TPW * D * 2);
-                vw[i] = *reinterpret_cast<const uint4*>(ks + Geo::PAGE_BYTES + (size_t)(i ^ xi) * TPW * D * 2);
+                    for (int h = 0; h < Geo::HALVES; ++h)
+                        if ((lane & 15) < 8)
+                            *reinterpret_cast<uint4*>(stage + (size_t)warp * Geo::PAGE_BYTES + Geo::BLOCK_BYTES + h * 2048 +
+                                                      r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                __syncwarp();
             }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty0 + 8 * s);
-
-        if (active) {
-            const bool tail = rows < (blk + 1) * kRowsPerWarp;
-            if (tail) {
+            // ---- S^T = K Q^T, two accumulators so that the MMAs are not one dependent chain
+            float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int i = 0; i < NR; ++i)
-                    if (blk * kRowsPerWarp + (i ^ xi) * TPW + grp >= rows) {
-                        kw[i] = make_uint4(0, 0, 0, 0);
-                        vw[i] = make_uint4(0, 0, 0, 0);
-                    }
+            for (int ks = 0; ks < Geo::KSTEPS; ++ks) {
+                const int piece = 2 * ks + k_piece;       // 16-byte piece of the row: half piece / 8
+                uint32_t a[4];
+                ldsm_x4(page_smem + (uint32_t)(piece >> 3) * 2048u + k_row + ((((uint32_t)piece & 7u) ^ k_swz) << 4), a);
+                if (ks & 1) mma_bf16(sb, a, qb[ks][0], qb[ks][1]);
+                else mma_bf16(sa, a, qb[ks][0], qb[ks][1]);
             }
-            // scores: partial dot products over this lane's 8 elements, then reduce over the row's lanes
-            float v[NV];
+            float sc[4];
 #pragma unroll
-            for (int i = 0; i < NR; ++i) {
-                const float2 k0 = unpack2(kw[i].x), k1 = unpack2(kw[i].y), k2 = unpack2(kw[i].z), k3 = unpack2(kw[i].w);
+            for (int e = 0; e < 4; ++e) sc[e] = (sa[e] + sb[e]) * qscale;      // log2 domain
+            // ---- mask: key key0 + g (+8) is visible to column c iff it lies below lim0 + token(c)
+            if (d.lim0 < key0 + kPage) {
+                const int lim_a = d.lim0 + (2 * t4) / G - key0, lim_b = d.lim0 + (2 * t4 + 1) / G - key0;
+                if (g >= lim_a) sc[0] = -INFINITY;
+                if (g >= lim_b) sc[1] = -INFINITY;
+                if (g + 8 >= lim_a) sc[2] = -INFINITY;
+                if (g + 8 >= lim_b) sc[3] = -INFINITY;
+            }
+            // ---- softmax against the lazily moved reference maxima of this thread's two columns
+            float c0 = fmaxf(sc[0], sc[2]), c1 = fmaxf(sc[1], sc[3]);
+            if (__any_sync(0xffffffffu, c0 > m0 + kRescaleThreshold || c1 > m1 + kRescaleThreshold)) {
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float2 a = __fmul2_rn(q2[g][0], k0);
-                    a = __ffma2_rn(q2[g][1], k1, a);
-                    a = __ffma2_rn(q2[g][2], k2, a);
-                    a = __ffma2_rn(q2[g][3], k3, a);
-                    v[i * G + g] = a.x + a.y;
+                for (int off = 4; off < 32; off <<= 1) {
+                    c0 = fmaxf(c0, __shfl_xor_sync(0xffffffffu, c0, off));
+                    c1 = fmaxf(c1, __shfl_xor_sync(0xffffffffu, c1, off));
+                }
+                const float n0 = fmaxf(m0, c0), n1 = fmaxf(m1, c1);
+                const float f0 = n0 == -INFINITY ? 1.f : fast_exp2(m0 - n0);
+                const float f1 = n1 == -INFINITY ? 1.f : fast_exp2(m1 - n1);
+                m0 = n0; m1 = n1;
+                l0 *= f0; l1 *= f1;
+#pragma unroll
+                for (int i = 0; i < Geo::KSTEPS; ++i) {
+                    o[i][0] *= f0; o[i][1] *= f1; o[i][2] *= f0; o[i][3] *= f1;
                 }
             }
-            transpose_reduce<NV, LPR / 2, NV>(v);
-            float sc[NF];
+            const float u0 = m0 == -INFINITY ? 0.f : m0, u1 = m1 == -INFINITY ? 0.f : m1;
+            const float p0 = fast_exp2(sc[0] - u0), p1 = fast_exp2(sc[1] - u1);
+            const float p2 = fast_exp2(sc[2] - u0), p3 = fast_exp2(sc[3] - u1);
+            l0 += p0 + p2;
+            l1 += p1 + p3;
+            // P (keys x columns, bf16) -> P^T as the B operand: two 8x8 transposes in registers
+            const uint32_t b0 = movmatrix_t(pack_bf16x2(p0, p1));
+            const uint32_t b1 = movmatrix_t(pack_bf16x2(p2, p3));
+            // ---- O^T += V^T P^T
 #pragma unroll
-            for (int f = 0; f < NF; ++f) sc[f] = v[f];
-            if (tail && blk * kRowsPerWarp + my_row >= rows) {
-#pragma unroll
-                for (int f = 0; f < NF; ++f) sc[f] = -INFINITY;
-            }
-            bool need = false;
-#pragma unroll
-            for (int f = 0; f < NF; ++f) need |= sc[f] > m_own[f] + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, need)) {
-                // move the reference maximum: per head, over this warp's rows of the tile
-                float mn[NF];
-#pragma unroll
-                for (int f = 0; f < NF; ++f) {
-                    float t = sc[f];
-                    t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 4));
-                    t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 8));
-                    t = fmaxf(t, __shfl_xor_sync(0xffffffffu, t, 16));
-                    mn[f] = fmaxf(m_own[f], t);
-                }
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const float mg = __shfl_xor_sync(0xffffffffu, mn[Geo::score_slot(0, g)], Geo::score_xor(0, g));
-                    const float scale = fast_exp2(m_ref[g] - mg);
-                    m_ref[g] = mg;
-                    const float2 s2 = make_float2(scale, scale);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) o2[g][j] = __fmul2_rn(o2[g][j], s2);
-                }
-#pragma unroll
-                for (int f = 0; f < NF; ++f) {
-                    l_own[f] *= fast_exp2(m_own[f] - mn[f]);
-                    m_own[f] = mn[f];
-                }
-            }
-            float pr[NF];
-#pragma unroll
-            for (int f = 0; f < NF; ++f) {
-                pr[f] = fast_exp2(sc[f] - m_own[f]);
-                l_own[f] += pr[f];
-            }
-#pragma unroll
-            for (int i = 0; i < NR; ++i) {
-                const float2 v0 = unpack2(vw[i].x), v1 = unpack2(vw[i].y), v2 = unpack2(vw[i].z), v3 = unpack2(vw[i].w);
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const float pg = __shfl_xor_sync(0xffffffffu, pr[Geo::score_slot(i, g)], Geo::score_xor(i, g));
-                    const float2 pp = make_float2(pg, pg);
-                    o2[g][0] = __ffma2_rn(pp, v0, o2[g][0]);
-                    o2[g][1] = __ffma2_rn(pp, v1, o2[g][1]);
-                    o2[g][2] = __ffma2_rn(pp, v2, o2[g][2]);
-                    o2[g][3] = __ffma2_rn(pp, v3, o2[g][3]);
-                }
+            for (int i = 0; i < Geo::KSTEPS; ++i) {
+                const int piece = 2 * i + v_piece;
+                uint32_t a[4];
+                ldsm_x4_t(page_smem + (uint32_t)(piece >> 3) * 2048u + v_row + ((((uint32_t)piece & 7u) ^ v_swz) << 4), a);
+                mma_bf16(o[i], a, b0, b1);
             }
         }
 
-        if (d.flags & kFlagLast) {
-            // ---- end of item: merge the warps' states and write the result
-            float* mm = merge_base + (size_t)(item_count & 1) * Geo::MERGE_FLOATS;   // [warp][G] max
-            float* ml = mm + Geo::STAT_FLOATS;                                    // [warp][G] sum
-            float* mo = ml + Geo::STAT_FLOATS;                                    // [warp][G][D]
+        if (!(d.flags & kFlagLast)) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * s);
+            continue;
+        }
+        // ---- end of item: merge the warps' states through this stage's shared memory (each warp's
+        // own page slot is free: only this warp read it) and write the result
+        {
+            float* st = reinterpret_cast<float*>(stage + (size_t)warp * Geo::PAGE_BYTES);
 #pragma unroll
-            for (int f = 0; f < NF; ++f) {
-                l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 4);
-                l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 8);
-                l_own[f] += __shfl_xor_sync(0xffffffffu, l_own[f], 16);
+            for (int off = 4; off < 32; off <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, off);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, off);
             }
+            __syncwarp();      // every lane is done reading the page before it is overwritten
 #pragma unroll
-            for (int off = LPR; off < 32; off <<= 1)
-#pragma unroll
-                for (int g = 0; g < G; ++g)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        o2[g][j].x += __shfl_xor_sync(0xffffffffu, o2[g][j].x, off);
-                        o2[g][j].y += __shfl_xor_sync(0xffffffffu, o2[g][j].y, off);
-                    }
-            if (grp == 0) {
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float4* dst = reinterpret_cast<float4*>(mo + ((size_t)warp * G + (g ^ xg)) * D + sub * 8);
-                    dst[0] = make_float4(o2[g][0].x, o2[g][0].y, o2[g][1].x, o2[g][1].y);
-                    dst[1] = make_float4(o2[g][2].x, o2[g][2].y, o2[g][3].x, o2[g][3].y);
-                }
-                if ((sub >> 2) == 0) {
-#pragma unroll
-                    for (int f = 0; f < NF; ++f) {
-                        const int k = NV >= LPR ? sub * NF + f : sub >> Geo::DUP_SHIFT;
-                        const int g = k % G;
-                        mm[warp * G + g] = m_own[f];
-                        ml[warp * G + g] = l_own[f];
-                    }
-                }
+            for (int i = 0; i < Geo::KSTEPS; ++i) {
+                float* c = st + (size_t)(2 * t4) * Geo::O_STRIDE + 16 * i + g;
+                c[0] = o[i][0];
+                c[Geo::O_STRIDE] = o[i][1];
+                c[8] = o[i][2];
+                c[Geo::O_STRIDE + 8] = o[i][3];
+            }
+            if (g == 0) {
+                float* ms = st + kCols * Geo::O_STRIDE;
+                ms[2 * t4] = m0; ms[2 * t4 + 1] = m1;
+                ms[kCols + 2 * t4] = l0; ms[kCols + 2 * t4 + 1] = l1;
             }
             __syncwarp();
-            const int buf = item_count & 1;
-            const uint32_t mb = mbar0 + 8 * buf;
-            if (lane == 0) mbar_arrive(mb);
-            // barrier `buf` serves every second item; its phase flips once per use
-            if (!mbar_wait(mb, (uint32_t)(item_count >> 1) & 1u, abort_flag, p.status, 3)) break;
+            if (lane == 0) mbar_arrive(mbar);
+            if (!mbar_wait(mbar, (uint32_t)item_count & 1u, abort_flag, p.status, 3)) break;
             ++item_count;
-            const int tid = threadIdx.x;
-            for (int e = 2 * tid; e < GT * D; e += 2 * kWarps * 32) {
-                const int gfull = e / D, dd = e % D;
-                const int g = gfull % G, w0 = (gfull / G) * RB;      // the RB warps that hold this head
+            const int ncols = cur_ntok * G;
+            for (int e = 2 * (int)threadIdx.x; e < ncols * D; e += 2 * kWarps * 32) {
+                const int col = e / D, dd = e % D;
                 float M = -INFINITY;
 #pragma unroll
-                for (int r = 0; r < RB; ++r) M = fmaxf(M, mm[(w0 + r) * G + g]);
+                for (int w = 0; w < kWarps; ++w)
+                    M = fmaxf(M, reinterpret_cast<const float*>(stage + (size_t)w * Geo::PAGE_BYTES)[kCols * Geo::O_STRIDE + col]);
                 float L = 0.f, a0 = 0.f, a1 = 0.f;
 #pragma unroll
-                for (int r = 0; r < RB; ++r) {
-                    const int w = w0 + r;
-                    const float wgt = fast_exp2(mm[w * G + g] - M);
-                    L = fmaf(ml[w * G + g], wgt, L);
-                    const float2 ov = *reinterpret_cast<const float2*>(mo + ((size_t)w * G + g) * D + dd);
-                    a0 = fmaf(ov.x, wgt, a0);
-                    a1 = fmaf(ov.y, wgt, a1);
+                for (int w = 0; w < kWarps; ++w) {
+                    const float* sw = reinterpret_cast<const float*>(stage + (size_t)w * Geo::PAGE_BYTES);
+                    const float mw = sw[kCols * Geo::O_STRIDE + col];
+                    const float wgt = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
+                    if (wgt != 0.f) {      // a warp without a visible key holds nothing worth reading
+                        L = fmaf(sw[kCols * Geo::O_STRIDE + kCols + col], wgt, L);
+                        const float2 ov = *reinterpret_cast<const float2*>(sw + (size_t)col * Geo::O_STRIDE + dd);
+                        a0 = fmaf(ov.x, wgt, a0);
+                        a1 = fmaf(ov.y, wgt, a1);
+                    }
                 }
-                const float inv = 1.f / L;
-                const size_t hq = (size_t)cur_kv_head * GT + gfull;
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+                const float lse2 = L > 0.f ? M + log2f(L) : -INFINITY;
+                const int tok = col / G, hh = col % G;
+                const size_t hq = (size_t)cur_kv_head * G + hh;
                 if (cur_partial < 0) {
-                    *reinterpret_cast<uint32_t*>(out + ((size_t)cur_out_row * Hq + hq) * D + dd) =
+                    *reinterpret_cast<uint32_t*>(out + ((size_t)(cur_out_row + tok) * Hq + hq) * D + dd) =
                         pack_bf16x2(a0 * inv, a1 * inv);
-                    if (lse != nullptr && dd == 0)
-                        lse[(size_t)cur_out_row * Hq + hq] = (M + log2f(L)) * kLn2;
+                    if (lse != nullptr && dd == 0) lse[(size_t)(cur_out_row + tok) * Hq + hq] = lse2 * kLn2;
                 } else {
-                    *reinterpret_cast<float2*>(p.partial_o + ((size_t)cur_partial * GT + gfull) * D + dd) =
+                    *reinterpret_cast<float2*>(p.partial_o + (((size_t)cur_partial + tok) * G + hh) * D + dd) =
                         make_float2(a0 * inv, a1 * inv);
-                    if (dd == 0) p.partial_lse[(size_t)cur_partial * GT + gfull] = M + log2f(L);
+                    if (dd == 0) p.partial_lse[((size_t)cur_partial + tok) * G + hh] = lse2;
                 }
             }
+            // the stage goes back to the producer, whose copies are writes of the asynchronous proxy
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * s);
         }
     }
 }

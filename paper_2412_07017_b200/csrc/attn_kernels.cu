@@ -11,6 +11,8 @@
 //   attn_decode_kernel     steps without span tiles, and head_dim 64
 // All are launched with programmatic stream serialization and wait for the kernel in front of them
 // (normally the KV append) right before they first touch the pool.
+#include <atomic>
+
 #include "attn_append_tc.cuh"
 #include "attn_decode.cuh"
 
@@ -30,7 +32,7 @@ attn_decode_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const 
                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
-    dec::decode_body<D, G, false>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw));
+    dec::decode_body<D, G>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw));
 }
 
 template <int G>
@@ -39,11 +41,11 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();      // the kernel behind this one may start its prologue; it waits for this grid to complete
-    tc::tc_body<G, false>(p, q, pool, out, lse, aligned_smem(smem_raw));
+    tc::tc_body<G>(p, q, pool, out, lse, aligned_smem(smem_raw));
 }
 
 template <int G>
-__global__ void __launch_bounds__(dec::kThreads, 1)
+__global__ void __launch_bounds__(tc::kThreads, 1)
 attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const __nv_bfloat16* __restrict__ q,
                   const __nv_bfloat16* __restrict__ pool, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                   int S) {
@@ -57,23 +59,25 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
     if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map));
     if (head[0] == head[1]) {
         // no span tiles for this CTA: straight to its decode rows, without the tensor-memory set-up
-        dec::decode_body<tc::kD, G, false>(p, &kv_map, q, out, lse, S, smem);
+        dec::decode_body<tc::kD, G>(p, &kv_map, q, out, lse, S, smem);
         return;
     }
-    tc::tc_body<G, true>(p, q, pool, out, lse, smem);
+    tc::tc_body<G>(p, q, pool, out, lse, smem);
     if (head[2] == head[3]) return;      // the planner gave this CTA its decode rows as tensor-core items too
     __syncthreads();      // tensor memory released, shared memory free for the second phase
-    dec::decode_body<tc::kD, G, true>(p, &kv_map, q, out, lse, S, smem);
+    dec::decode_body<tc::kD, G>(p, &kv_map, q, out, lse, S, smem);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// The pool as a 5-D tensor (d, 16 slots, Hkv, K|V, pages) with a box of one page's K and V blocks of
-// one kv head (see dec::tma_page_kv).  The driver entry point is looked up once per process.
+// The pool as a 5-D tensor (64 values, 16 slots, d / 64 row halves, Hkv, pages x K|V) with a box of
+// one page's K and V blocks of one kv head, landed with the 128-byte swizzle (see dec::tma_page_kv).
+// The driver entry point is looked up once per process.
 cudaError_t make_kv_map(const DevPlan& p, const void* pool, CUtensorMap* map) {
-    static EncodeTiledFn encode = nullptr;
+    static std::atomic<EncodeTiledFn> encode_fn{nullptr};
+    EncodeTiledFn encode = encode_fn.load(std::memory_order_acquire);
     if (encode == nullptr) {
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -81,31 +85,32 @@ cudaError_t make_kv_map(const DevPlan& p, const void* pool, CUtensorMap* map) {
         if (e != cudaSuccess) return e;
         if (qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
         encode = (EncodeTiledFn)sym;
+        encode_fn.store(encode, std::memory_order_release);
     }
     const cuuint64_t d = (cuuint64_t)p.head_dim, hkv = (cuuint64_t)p.num_kv_heads;
-    if (p.num_pages <= 0 || p.num_pages > 0x7fffffff) return cudaErrorInvalidValue;
-    const cuuint64_t dims[5] = {d, kPage, hkv, 2, (cuuint64_t)p.num_pages};
-    const cuuint64_t strides[4] = {d * 2, kPage * d * 2, hkv * kPage * d * 2, 2 * hkv * kPage * d * 2};
-    const cuuint32_t box[5] = {(cuuint32_t)d, kPage, 1, 2, 1};
+    if (p.num_pages <= 0 || p.num_pages > 0x3fffffff) return cudaErrorInvalidValue;
+    const cuuint64_t dims[5] = {64, kPage, d / 64, hkv, 2 * (cuuint64_t)p.num_pages};
+    const cuuint64_t strides[4] = {d * 2, 128, kPage * d * 2, hkv * kPage * d * 2};
+    const cuuint32_t box[5] = {64, kPage, (cuuint32_t)(d / 64), 1, 2};
     const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
     const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box,
-                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-template <int D, int G>
+template <int D>
 int decode_stages() {
-    int S = 8;
-    while (S > 2 && dec::smem_bytes<D, G>(S) > (size_t)kMaxSmem) --S;
+    int S = 6;
+    while (S > 2 && dec::smem_bytes<D>(S) > (size_t)kMaxSmem) --S;
     return S;
 }
 
 template <int D, int G>
 cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                           cudaStream_t stream) {
-    const int S = decode_stages<D, G>();
-    const size_t smem = dec::smem_bytes<D, G>(S);
+    const int S = decode_stages<D>();
+    const size_t smem = dec::smem_bytes<D>(S);
     cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
@@ -128,14 +133,14 @@ cudaError_t launch_tensor(const DevPlan& p, const void* q, const void* pool, voi
 template <int G>
 cudaError_t launch_fused(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                          cudaStream_t stream) {
-    const int S = decode_stages<tc::kD, G>();
-    const size_t smem = dec::smem_bytes<tc::kD, G>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD, G>(S) : tc::kSmemBytes;
+    const int S = decode_stages<tc::kD>();
+    const size_t smem = dec::smem_bytes<tc::kD>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD>(S) : tc::kSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
     e = make_kv_map(p, pool, &map);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_fused_kernel<G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p, map,
+    return launch_pdl(attn_fused_kernel<G>, dim3(p.num_ctas_cuda), dim3(tc::kThreads), smem, stream, p, map,
                       (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S);
 }
 

@@ -225,7 +225,7 @@ struct PathCost {
 };
 // (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
 constexpr PathCost kTensorCost{128, 1170, 8000, 11800};
-constexpr PathCost kCudaCost{96, 1280, 1200, 5000};
+constexpr PathCost kCudaCost{128, 900, 1200, 2000};
 constexpr int64_t kTensorDualTileNs = 2435;   // a KV tile of an item with two row tiles (more than 128 rows)
 // When every unit runs on the tensor-core kernel all SMs stream K/V tiles at once and the tile time is
 // set by the memory system (64 KB per tile and SM: 148 SMs at 37 KB/us are 5.5 TB/s); the producers
@@ -256,12 +256,6 @@ void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& id
     // a narrow item (one decode token's rows) on the tensor-core body: tile and item cost
     const int64_t narrow_tile_ns = tensor_only ? kTensorOnlyCost.tile_ns : 1400;
     const int64_t narrow_item_ns = 2900;
-    if (group > 4) {
-        // 8 heads per kv head: the decode kernel runs two head halves over 48-key tiles and is bound by
-        // its arithmetic; measured 2.42 us per 96 keys and 1.4 us per item on the 64/8-head batch
-        cost[1].tile_ns = 2420;
-        cost[1].item_ns = 1400;
-    }
     auto tile_ns = [&](int path, int id) {
         return path == 0 && units[id].u.ntok * group > 128 ? dual_tile_ns : cost[path].tile_ns;
     };
