@@ -31,9 +31,9 @@ METRIC = "kv_gbps_mixed_decode_interrupt_append"
 UNIT = "GB/s"
 WORKLOAD = "config2-llama3-8b-mixed-batch"       # the configuration the metric is quoted on (default)
 WORKLOADS = {2: WORKLOAD, 3: "config3-large-batch-gqa8", 4: "config4-long-context-split-kv"}
-# dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on this workload
-# (profiles/attn_fused_kernel_config2.md); None whenever the kernel has changed since that capture
-TRAFFIC_BYTES_PER_LAUNCH = 327_827_712
+# dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on the default
+# workload, from an ncu capture; None whenever the kernel has changed since the counters were taken
+TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def measured_peaks():
@@ -93,6 +93,23 @@ class ClockSampler:
                           if v.lower().startswith("active")})
         return {"sm_mhz": float(np.median([s[1] for s in inside])), "sm_max_mhz": inside[0][2],
                 "reasons": reasons, "samples": len(inside)}
+
+
+class L2Flush:
+    """Evicts the KV pool from L2 between timed steps (untimed): a 256 MiB buffer is rewritten, which
+    pushes everything else out, and then another 256 MiB buffer is read, which leaves L2 full of
+    clean lines.  Without the read pass L2 would still hold up to 126 MB of the fill's dirty lines,
+    and their write-back would ride on the timed step's DRAM traffic (measured: 17 us of a 107 us
+    decode-only step)."""
+    NOTE = "256 MiB buffer rewritten, then a second 256 MiB buffer read, between timed steps (untimed)"
+
+    def __init__(self, torch):
+        self.w = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > 126 MB L2
+        self.r = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")
+
+    def fill_(self, v):
+        self.w.fill_(v)
+        self.r.sum()
 
 
 # ------------------------------------------------------------------------------------------------
@@ -184,7 +201,7 @@ def run_gpu(args):
 
     if args.decode_only:
         # 64 sequences of the Llama-3-8B attention shape, contexts uniform in [1024, 3072], one decode
-        # token each: the CUDA-core decode kernel alone (profiling aid, not the benchmarked workload)
+        # token each: the warp body alone (profiling aid, not the benchmarked workload)
         lens = np.random.default_rng(3).integers(1024, 3073, 64).tolist()
         wl = W.make_single_step("decode-only", W.Shape(32, 8, 128, 16), lens, [1] * 64, seed=11)
     elif args.spans_only:
@@ -206,7 +223,7 @@ def run_gpu(args):
     q, kn, vn = dev(st.q), dev(st.k_new), dev(st.v_new)
     T = st.total_q
     out = torch.empty((T, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > 126 MB L2
+    flush = L2Flush(torch)
     stream = torch.cuda.current_stream()
 
     hb, db = B.workspace_size(shape, wl.num_pages, st.batch, T, len(st.page_indices))
@@ -347,7 +364,7 @@ def run_gpu(args):
                         "spans-only-24x[1024,3072]+64" if args.spans_only else WORKLOADS[args.config],
             "seed": wl.seed, "batch": st.batch, "total_q": T,
             "kv_tokens": int(plan.info["total_kv_tokens"]), "replicas": world,
-            "l2": "256 MiB buffer rewritten between timed steps (untimed)",
+            "l2": L2Flush.NOTE,
             "us_per_step": ms_per_step * 1e3,
             "us_per_step_without_l2_flush": float(np.median(noflush_ms)) * 1e3,
             "us_per_step_p10_p50_p90": [float(np.percentile(step_ms, p)) * 1e3 for p in (10, 50, 90)],
@@ -404,7 +421,7 @@ def run_replay(args):
     dq = [(dev(st.q), dev(st.k_new), dev(st.v_new)) for st in steps]
     max_T = max(st.total_q for st in steps)
     out = torch.empty((max_T, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = L2Flush(torch)
     stream = torch.cuda.current_stream()
     hb, db = B.workspace_size(shape, wl.num_pages, steps[0].batch, max_T,
                               max(len(st.page_indices) for st in steps))
@@ -447,7 +464,7 @@ def run_replay(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {
             "workload": "config5-interrupt-trace-replay", "seed": wl.seed, "batch": steps[0].batch,
-            "l2": "256 MiB buffer rewritten between timed steps (untimed)",
+            "l2": L2Flush.NOTE,
             "us_per_step_first_median_last": [float(dev_us[0]), float(np.median(dev_us)), float(dev_us[-1])],
             "us_per_step_p10_p90": [float(np.percentile(dev_us, 10)), float(np.percentile(dev_us, 90))],
             "us_per_step_with_interrupts": float(dev_us[np.array(spans) > 0].mean()) if any(spans) else None,

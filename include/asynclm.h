@@ -73,19 +73,18 @@ typedef struct asynclm_plan_options {
     int32_t kv_chunk_tokens;  /* fixed split-KV chunk length (multiple of 64); 0 = chosen so that
                                  the work items roughly fill the machine; a value >= the longest
                                  context disables splitting */
-    int32_t tensor_min_rows;  /* new tokens of a sequence use the tensor-core path when
-                                 G * q_len >= this; 0 = default: 32 for G <= 4 (a decode row
-                                 then runs on the CUDA-core path, except on a CTA that also
-                                 holds span tiles, where it runs as a narrow tensor-core item),
-                                 and 8 for G = 8, where the CUDA-core path is bound by its
-                                 arithmetic rather than by memory;
-                                 INT32_MAX keeps every row on the CUDA-core path, like
-                                 ASYNCLM_PLAN_NO_TENSOR_PATH */
+    int32_t tensor_min_rows;  /* new tokens of a sequence use the span body (tcgen05 MMA, 128
+                                 query rows to a tile) when G * q_len >= this; 0 = default: 32.
+                                 Below it they use the warp body (warp-level MMA with the keys
+                                 on the M axis, 8 / G tokens to a unit), which streams K/V at
+                                 the memory rate for every supported G and is where decode
+                                 rows always go by default.  INT32_MAX keeps every row on the
+                                 warp body, like ASYNCLM_PLAN_NO_TENSOR_PATH */
     int32_t flags;            /* ASYNCLM_PLAN_* */
 } asynclm_plan_options;
 
 #define ASYNCLM_PLAN_REJECT_ALIASED_WRITES 1  /* error if two sequences append into one page */
-#define ASYNCLM_PLAN_NO_TENSOR_PATH        2  /* keep every row on the CUDA-core path         */
+#define ASYNCLM_PLAN_NO_TENSOR_PATH        2  /* keep every row on the warp body              */
 
 /* Host-side description of one step's batch (all arrays on the host, int32). */
 typedef struct asynclm_batch {
@@ -111,9 +110,9 @@ typedef struct asynclm_plan_info {
     int32_t num_split_units;  /* units whose keys were split into > 1 chunk */
     int32_t partial_rows;     /* rows of fp32 partial output held in the device workspace */
     int32_t kv_chunk_tokens;  /* chosen chunk length (INT32_MAX = unsplit) */
-    int32_t num_ctas_cuda;    /* persistent CTAs of the CUDA-core attention kernel */
-    int32_t num_ctas_tensor;  /* persistent CTAs of the tensor-core attention kernel */
-    int32_t num_items_tensor; /* items routed to the tensor-core kernel */
+    int32_t num_ctas_cuda;    /* persistent CTAs that may run the warp body */
+    int32_t num_ctas_tensor;  /* persistent CTAs that may run the span body */
+    int32_t num_items_tensor; /* items routed to the span body */
     int32_t launches_append;  /* kernels asynclm_kv_append launches */
     int32_t launches_attn;    /* kernels asynclm_attn_mixed launches */
     int32_t num_sms;
@@ -129,14 +128,16 @@ typedef struct asynclm_item_view {
     int32_t tok0;       /* first new token of the unit, index i inside the sequence's span */
     int32_t ntok;       /* tokens of the span covered by the unit */
     int32_t kv0, kv1;   /* key positions [kv0, kv1) the item reads (before causal clipping) */
-    int32_t path;       /* 0 = CUDA-core kernel, 1 = tensor-core kernel */
-    int32_t cta;        /* persistent CTA (within its kernel) that processes the item */
+    int32_t path;       /* 0 = warp body, 1 = span body */
+    int32_t cta;        /* persistent CTA that processes the item; -1 = handed out at run time to
+                           whichever CTA is free (items are listed in hand-out order) */
 } asynclm_item_view;
 
 int asynclm_version(void);
 const char* asynclm_strerror(int status);
 /* Text of the CUDA error behind the calling thread's most recent ASYNCLM_ERR_CUDA from
-   asynclm_kv_append / asynclm_attn_mixed ("no error" if there was none). */
+   asynclm_kv_append / asynclm_attn_mixed / asynclm_attn_mixed_static ("no error" if there was
+   none). */
 const char* asynclm_last_cuda_error(void);
 
 /*
@@ -153,13 +154,21 @@ int asynclm_plan_workspace_size(const asynclm_shape* shape, const asynclm_plan_o
  *
  * Validates the batch, tiles every (sequence, kv head) into query tiles and page-aligned KV chunks
  * (long contexts are split; partial results are merged by log-sum-exp inside asynclm_attn_mixed),
- * assigns the items to persistent CTAs under the smallest per-CTA load limit that fits (span tiles
- * are kept whole where possible, largest first; decode rows fill the CTAs up and are cut only
- * where a CTA is full; a CTA runs one kernel body only, so decode rows placed beside span tiles
- * become tensor-core items), then enqueues ONE host->device copy of the packed plan on `stream`.
+ * and decides who runs what: span tiles are packed whole where possible, largest first, onto as
+ * few persistent CTAs as a load limit allows (a span of two row tiles that does not fit is divided
+ * by rows before it is cut by keys); decode rows and short spans are cut into chunks (long pieces
+ * first, short ones from a few units at the end) that the CTAs take from a queue at run time, one
+ * atomic add per chunk, so that no cost model has to predict how fast each SM streams.  Results do
+ * not depend on which CTA ran which chunk: partial results are indexed by chunk and merged in
+ * chunk order.  Then ONE host->device copy of the packed plan is enqueued on `stream`.
  *
- *   host_ws / host_bytes  host memory (8-byte aligned; pinned recommended) that must stay untouched
- *                         until the copy has completed and for as long as the plan is used.
+ * A plan holds a few counters in its device workspace (queue position, arrivals per split unit)
+ * that every launch leaves at zero; launches that use the same plan must therefore not overlap on
+ * the GPU (use one stream, as the layers of a model do, or order them with events).
+ *
+ *   host_ws / host_bytes  host memory (16-byte aligned; pinned recommended) that must stay
+ *                         untouched until the copy has completed and for as long as the plan is
+ *                         used.
  *   dev_ws / dev_bytes    device memory (256-byte aligned) owned by the caller.  dev_ws == NULL
  *                         builds the plan on the host only (no CUDA call is made; opts->num_sms
  *                         must be set); such a plan can be inspected but not executed.
@@ -205,7 +214,8 @@ int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, const void*
  *   q    device, bf16 [T][num_q_heads][head_dim]
  *   out  device, bf16 [T][num_q_heads][head_dim]
  *   lse  device, fp32 [T][num_q_heads], natural log; may be NULL
- * Errors: INVALID_ARG, CUDA.
+ * The current device must be the one the plan was made on.
+ * Errors: INVALID_ARG (also: another device is current), CUDA.
  */
 int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv_pool,
                        void* out, float* lse, void* stream);
@@ -240,7 +250,8 @@ int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t
  *     kv_chunk_tokens, or use asynclm_attn_mixed.
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress with that device current).  Make that first call before starting any
- *     stream capture on that device.
+ *     stream capture on that device, and while the device still has the array's size to spare: the
+ *     driver may set the library image's data up only then.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left in
  *     it.  Nothing in it has to start at zero: each call writes every partial row before reading
  *     it.  Two calls whose kernels may overlap on the GPU (different streams, or different threads

@@ -77,8 +77,8 @@ def load(rebuild_if_stale: bool = True):
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
-    if rebuild_if_stale and _build.find_nvcc() is not None and _build.is_stale():
+    path = os.environ.get("ASYNCLM_LIBRARY") or _build.LIB      # e.g. the time-stamp build of build.py
+    if path == _build.LIB and rebuild_if_stale and _build.find_nvcc() is not None and _build.is_stale():
         _build.build()
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing and could not be built; the CUDA library is required "

@@ -11,6 +11,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(CSRC, "libasynclm.so")
+# A second build with per-CTA time stamps compiled in (-DASYNCLM_TRACE, asynclm_trace_read): for
+# performance work only; the binding loads it when ASYNCLM_LIBRARY points at it.
+TRACE_LIB = os.path.join(CSRC, "libasynclm_trace.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -39,23 +42,24 @@ def find_nvcc():
     return nvcc if os.path.exists(nvcc) else None
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not is_stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+    lib = TRACE_LIB if trace else LIB
+    if not force and not trace and not is_stale():
+        return lib
     nvcc = find_nvcc()
     if nvcc is None:
         raise RuntimeError("nvcc not found; cannot build libasynclm.so")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-        ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
+        (["-DASYNCLM_TRACE"] if trace else []) + ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + proc.stdout + proc.stderr)
     if verbose:
         sys.stderr.write(proc.stderr)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))

@@ -9,11 +9,18 @@ using namespace asynclm;
 
 static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
 
-static int cuda_status(cudaError_t e) {
+int asynclm::cuda_status(cudaError_t e) {
     if (e == cudaSuccess) return ASYNCLM_OK;
     g_last_cuda_error = e;
     (void)cudaGetLastError();   // clear the sticky launch-configuration error, if that is what it was
     return ASYNCLM_ERR_CUDA;
+}
+
+int asynclm::check_plan_device(int plan_device) {
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_status(e);
+    return dev == plan_device ? ASYNCLM_OK : ASYNCLM_ERR_INVALID_ARG;
 }
 
 extern "C" int asynclm_version(void) { return 100; }
@@ -48,6 +55,7 @@ extern "C" int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, 
     if (plan->dev.total_q == 0) return ASYNCLM_OK;
     if (!k_new || !v_new || !kv_pool || !aligned16(k_new) || !aligned16(v_new) || !aligned16(kv_pool))
         return ASYNCLM_ERR_INVALID_ARG;
+    if (int rc = check_plan_device(plan->device)) return rc;
     return cuda_status(launch_kv_append(plan->dev, k_new, v_new, kv_pool, (cudaStream_t)stream));
 }
 
@@ -57,6 +65,7 @@ extern "C" int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, con
     if (plan->dev.total_q == 0) return ASYNCLM_OK;
     if (!q || !kv_pool || !out || !aligned16(q) || !aligned16(kv_pool) || !aligned16(out))
         return ASYNCLM_ERR_INVALID_ARG;
+    if (int rc = check_plan_device(plan->device)) return rc;
     cudaStream_t s = (cudaStream_t)stream;
     int rc = cuda_status(launch_attention(plan->dev, q, kv_pool, out, lse, s));
     if (rc != ASYNCLM_OK) return rc;

@@ -20,9 +20,13 @@
 // travel with each stage.  Eight consumer warps take one page of a stage each: ldmatrix, the two
 // contractions, softmax against a lazily moved reference maximum on the accumulator fragment
 // (4 values per thread), P transposed in registers (movmatrix) into the B operand.  At the end of
-// an item the warps' states are merged through the shared memory of the item's last stage (which
-// is idle by then) and written either as final bf16 output or as an fp32 partial for the split-KV
-// merge.
+// an item each consumer warp drops its state into its own page slot of the item's last stage and
+// goes straight on to the next item; an epilogue warp combines the eight states, writes final bf16
+// output or the fp32 partial of a chunk, and hands the stage back to the producer.  When the chunk
+// belongs to a unit whose keys were split, the epilogue warp also counts it in (one atomic add per
+// chunk); the CTA that brings the count to the number of chunks merges the unit's partial results
+// in chunk order on a merge warp of its own, so no merge kernel has to follow and no consumer ever
+// waits for another warp.
 //
 // Every wait is bounded: a wait that runs out sets the plan's device status word and a CTA-wide
 // abort flag, after which all loops fall through and the kernel returns.
@@ -38,7 +42,13 @@ namespace dec {
 
 constexpr int kWarps = 8;                    // consumer warps: one page of a 128-key stage each
 constexpr int kProducerWarp = kWarps;        // the warp behind them streams the pages
-constexpr int kThreads = (kWarps + 2) * 32;  // standalone kernel: consumers, producer, one spare warp
+constexpr int kEpilogueWarp = kWarps + 1;    // combines the consumers' states at the end of an item
+constexpr int kMergeWarp = kWarps + 2;       // merges the chunks of a split unit once all have arrived
+constexpr int kFetchWarp = kWarps + 3;       // claims the next chunk and fetches its record and page ids
+constexpr int kThreads = (kWarps + 4) * 32;  // consumers, producer, epilogue, merge, fetch
+constexpr int kMergeReqs = 4;                // merge requests in flight between the last two
+constexpr int kMaxStages = 6;
+constexpr int kHandoffs = kMaxStages + 2;    // item hand-offs in flight: a stage each, so at most kMaxStages
 constexpr int kCols = 8;                     // (token, head) columns of a unit: the N of the MMAs
 constexpr int kTileTok = kWarps * kPage;     // keys per ring stage
 constexpr float kRescaleThreshold = 8.f;     // log2 units a score may exceed the reference max by
@@ -54,7 +64,17 @@ struct TileDesc {
     int32_t out_row;      // global token row of the unit's first token
     int32_t kv_head;
     int32_t partial_row;  // -1: final output
+    int32_t unit;         // the unit the item is a chunk of, its number of chunks and the partial row of
+    int32_t n_chunks;     // its chunk 0 (for the merge of a split unit)
+    int32_t partial_base;
+    int32_t stage;        // hand-off only: the stage that holds the consumers' states
     int32_t pad;
+};
+
+// What the fetch warp hands to the producer: the next item's record and its first 32 page ids.
+struct NextItem {
+    int32_t work[12];     // a Work record; work[1] (kv_end) == 0: nothing is left
+    int32_t pages[32];
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -65,6 +85,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -158,11 +181,193 @@ struct Geometry {
 template <int D>
 size_t smem_bytes(int stages) {
     using Geo = Geometry<D>;
-    return (size_t)stages * (Geo::STAGE_BYTES + Geo::Q_BYTES + sizeof(TileDesc) + 16) + 8 + 16 + 1024;
+    return (size_t)stages * (Geo::STAGE_BYTES + Geo::Q_BYTES + sizeof(TileDesc) + 16) +
+           (size_t)(kHandoffs + kMergeReqs) * (sizeof(TileDesc) + 8) + kMergeReqs * 8 + sizeof(NextItem) + 16 +
+           16 + 1024;
 }
 
-// The whole kernel body: warps 0-7 consume, warp 8 produces, any further warps of the CTA return at
-// once (the fused kernel has twelve).
+// The epilogue warp's loop (see the file comment): combine the consumers' states of a finished item,
+// write the result, give the stage back, and pass a completed split unit on to the merge warp.
+template <int D, int G>
+__device__ __forceinline__ void epilogue_loop(const DevPlan& p, __nv_bfloat16* __restrict__ out,
+                                              float* __restrict__ lse, uint8_t* stage_base,
+                                              const TileDesc* handoff, TileDesc* merge_req, uint32_t empty0,
+                                              uint32_t done0, uint32_t req0, uint32_t reqfree0,
+                                              volatile int* abort_flag) {
+    using Geo = Geometry<D>;
+    const int lane = threadIdx.x & 31;
+    const int Hq = p.num_q_heads;
+    int n_req = 0;
+    auto post = [&](const TileDesc& d) {      // to the merge warp; false if the wait for a free slot ran out
+        const int j = n_req % kMergeReqs;
+        if (!mbar_wait(reqfree0 + 8 * j, ((uint32_t)(n_req / kMergeReqs) & 1u) ^ 1u, abort_flag, p.status, 4)) return false;
+        if (lane == 0) {
+            merge_req[j] = d;
+            mbar_arrive(req0 + 8 * j);
+        }
+        ++n_req;
+        return true;
+    };
+    pdl_wait();      // outputs may be written only after the kernel in front has completed
+    for (int k = 0;; ++k) {
+        const int h = k % kHandoffs;
+        if (!mbar_wait(done0 + 8 * h, (uint32_t)(k / kHandoffs) & 1u, abort_flag, p.status, 3)) break;
+        const TileDesc d = handoff[h];
+        if (d.flags & kFlagEnd) {
+            post(d);
+            break;
+        }
+        const uint8_t* stage = stage_base + (size_t)d.stage * Geo::STAGE_BYTES;
+        const int ncols = d.ntok * G;
+        // four consecutive values of one column per lane and pass; the eight warps' copies are read
+        // with independent loads
+        for (int e = 4 * lane; e < ncols * D; e += 128) {
+            const int col = e / D, dd = e % D;
+            float mw[kWarps], lw[kWarps];
+            float4 ov[kWarps];
+            float M = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float* sw = reinterpret_cast<const float*>(stage + (size_t)w * Geo::PAGE_BYTES);
+                mw[w] = sw[kCols * Geo::O_STRIDE + col];
+                lw[w] = sw[kCols * Geo::O_STRIDE + kCols + col];
+                ov[w] = *reinterpret_cast<const float4*>(sw + (size_t)col * Geo::O_STRIDE + dd);
+                M = fmaxf(M, mw[w]);
+            }
+            float L = 0.f;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float wgt = mw[w] == -INFINITY ? 0.f : fast_exp2(mw[w] - M);
+                if (wgt != 0.f) {      // a warp without a visible key left nothing meaningful behind
+                    L = fmaf(lw[w], wgt, L);
+                    a.x = fmaf(ov[w].x, wgt, a.x); a.y = fmaf(ov[w].y, wgt, a.y);
+                    a.z = fmaf(ov[w].z, wgt, a.z); a.w = fmaf(ov[w].w, wgt, a.w);
+                }
+            }
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+            const float lse2 = L > 0.f ? M + log2f(L) : -INFINITY;
+            const int tok = col / G, hh = col % G;
+            const size_t hq = (size_t)d.kv_head * G + hh;
+            if (d.partial_row < 0) {
+                *reinterpret_cast<uint2*>(out + ((size_t)(d.out_row + tok) * Hq + hq) * D + dd) =
+                    make_uint2(pack_bf16x2(a.x * inv, a.y * inv), pack_bf16x2(a.z * inv, a.w * inv));
+                if (lse != nullptr && dd == 0) lse[(size_t)(d.out_row + tok) * Hq + hq] = lse2 * kLn2;
+            } else {
+                *reinterpret_cast<float4*>(p.partial_o + (((size_t)d.partial_row + tok) * G + hh) * D + dd) =
+                    make_float4(a.x * inv, a.y * inv, a.z * inv, a.w * inv);
+                if (dd == 0) p.partial_lse[((size_t)d.partial_row + tok) * G + hh] = lse2;
+            }
+        }
+        // the stage goes back to the producer (whose copies are writes of the asynchronous proxy) on
+        // behalf of the eight consumer warps
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive_n(empty0 + 8 * d.stage, kWarps);
+        if (d.partial_row < 0) continue;
+        // ---- a chunk of a split unit: count it in; the CTA that completes the unit merges it
+        __threadfence();      // this warp's partial rows are visible device-wide before the count moves
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) last = atomicAdd(p.unit_arrivals + d.unit, 1) == d.n_chunks - 1;
+        if (__shfl_sync(0xffffffffu, last, 0) && !post(d)) break;
+    }
+}
+
+// The merge warp's loop: LSE = log sum_c exp(LSE_c), O = sum_c exp(LSE_c - LSE) O_c over the chunks
+// of a completed split unit, in chunk order.  All chunks are read back from memory (this CTA's own
+// included), so the result does not depend on which CTA finished the unit.
+template <int D, int G>
+__device__ __forceinline__ void merge_loop(const DevPlan& p, __nv_bfloat16* __restrict__ out,
+                                           float* __restrict__ lse, const TileDesc* merge_req,
+                                           uint32_t req0, uint32_t reqfree0, volatile int* abort_flag) {
+    const int lane = threadIdx.x & 31;
+    const int Hq = p.num_q_heads;
+    pdl_wait();
+    for (int k = 0;; ++k) {
+        const int j = k % kMergeReqs;
+        if (!mbar_wait(req0 + 8 * j, (uint32_t)(k / kMergeReqs) & 1u, abort_flag, p.status, 5)) break;
+        const TileDesc d = merge_req[j];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(reqfree0 + 8 * j);
+        if (d.flags & kFlagEnd) break;
+        __threadfence();      // the chunks' rows were written before their counts moved: visible now
+        const int ncols = d.ntok * G;
+        // four consecutive values of one column per lane and position, two positions at a time and up
+        // to eight chunks per pass, all requested together: one round trip to L2 per pass
+        for (int e0 = 4 * lane; e0 < ncols * D; e0 += 256) {
+            float4 acc[2];
+            float mx[2], wsum[2];
+            size_t prow0[2], hh[2];
+            int dd[2];
+            bool on[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int e = e0 + 128 * u;
+                on[u] = e < ncols * D;
+                const int col = on[u] ? e / D : 0;
+                dd[u] = e % D;
+                hh[u] = (size_t)(col % G);
+                prow0[u] = (size_t)d.partial_base + col / G;       // chunk c -> prow0 + c * ntok
+                acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                mx[u] = -INFINITY;
+                wsum[u] = 0.f;
+            }
+            for (int c0 = 0; c0 < d.n_chunks; c0 += 8) {
+                float l2[2][8];
+                float4 v[2][8];
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        l2[u][i] = -INFINITY;
+                        v[u][i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (on[u] && c0 + i < d.n_chunks) {
+                            const size_t r = (prow0[u] + (size_t)(c0 + i) * d.ntok) * G + hh[u];
+                            l2[u][i] = __ldcg(p.partial_lse + r);
+                            v[u][i] = __ldcg(reinterpret_cast<const float4*>(p.partial_o + r * D + dd[u]));
+                        }
+                    }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    float pm = mx[u];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) pm = fmaxf(pm, l2[u][i]);
+                    const float rescale = pm == -INFINITY ? 1.f : fast_exp2(mx[u] - pm);      // first pass: exp2(-inf) = 0
+                    mx[u] = pm;
+                    wsum[u] *= rescale;
+                    acc[u].x *= rescale; acc[u].y *= rescale; acc[u].z *= rescale; acc[u].w *= rescale;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float w = l2[u][i] == -INFINITY ? 0.f : fast_exp2(l2[u][i] - mx[u]);   // -inf: no visible key there
+                        wsum[u] += w;
+                        if (w != 0.f) {
+                            acc[u].x = fmaf(w, v[u][i].x, acc[u].x); acc[u].y = fmaf(w, v[u][i].y, acc[u].y);
+                            acc[u].z = fmaf(w, v[u][i].z, acc[u].z); acc[u].w = fmaf(w, v[u][i].w, acc[u].w);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if (!on[u]) continue;
+                const int col = (e0 + 128 * u) / D, tok = col / G;
+                const float inv = 1.f / wsum[u];
+                const size_t hq = (size_t)d.kv_head * G + hh[u];
+                *reinterpret_cast<uint2*>(out + ((size_t)(d.out_row + tok) * Hq + hq) * D + dd[u]) =
+                    make_uint2(pack_bf16x2(acc[u].x * inv, acc[u].y * inv), pack_bf16x2(acc[u].z * inv, acc[u].w * inv));
+                if (lse != nullptr && dd[u] == 0)
+                    lse[(size_t)(d.out_row + tok) * Hq + hq] = (mx[u] + log2f(wsum[u])) * kLn2;
+            }
+        }
+        if (lane == 0) atomicExch(p.unit_arrivals + d.unit, 0);      // ready for the next launch of this plan
+        if (lane == 0) trace_add(7, 1);
+    }
+    if (lane == 0) trace_mark(3);
+}
+
+// The whole kernel body: warps 0-7 consume, warp 8 produces, warps 9 and 10 are the epilogue and the
+// merge warp, any further warps of the CTA return at once (the fused kernel has twelve).
 template <int D, int GT>
 __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap* kv_map,
                                             const __nv_bfloat16* __restrict__ q,
@@ -174,12 +379,17 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
     uint8_t* stage_base = smem;                                        // 1024-byte aligned
     uint8_t* q_base = stage_base + (size_t)S * Geo::STAGE_BYTES;
     TileDesc* desc = (TileDesc*)(q_base + (size_t)S * Geo::Q_BYTES);
-    uint64_t* bars = (uint64_t*)(desc + S);      // full[S], empty[S], merge
-    volatile int* abort_flag = (volatile int*)(bars + 2 * S + 1);
+    TileDesc* handoff = desc + S;                // what the epilogue warp needs to know about a finished item
+    TileDesc* merge_req = handoff + kHandoffs;   // completed split units on their way to the merge warp
+    NextItem* next_item = (NextItem*)(merge_req + kMergeReqs);
+    uint64_t* bars = (uint64_t*)(next_item + 1);   // full[S], empty[S], done[kHandoffs], req, reqfree, next full, free
+    volatile int* abort_flag = (volatile int*)(bars + 2 * S + kHandoffs + 2 * kMergeReqs + 2);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), mbar = smem_u32(bars + 2 * S);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + S), done0 = smem_u32(bars + 2 * S);
+    const uint32_t req0 = done0 + 8 * kHandoffs, reqfree0 = req0 + 8 * kMergeReqs;
+    const uint32_t next_full = reqfree0 + 8 * kMergeReqs, next_free = next_full + 8;
 
     if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(kv_map));
     if (threadIdx.x == 0) {
@@ -187,7 +397,8 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, kWarps);
         }
-        mbar_init(mbar, kWarps);
+        for (int h = 0; h < kHandoffs; ++h) mbar_init(done0 + 8 * h, kWarps);
+        for (int j = 0; j < 2 * kMergeReqs + 2; ++j) mbar_init(req0 + 8 * j, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -196,26 +407,21 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
 
     const int Hq = p.num_q_heads;
 
-    if (warp >= kWarps) {
-        if (warp != kProducerWarp) return;      // spare warps have nothing to do
+    if (warp > kFetchWarp) return;      // further warps of the CTA have nothing to do
+    if (warp == kProducerWarp) {
         // ------------------------------------------------------------------ producer warp
-        // The page ids of the next 32 pages (4 stages) and the descriptors of the next two items are
-        // fetched ahead of use, so that no global-load latency sits between two stages.
-        struct PItem { int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row, page0; };
+        // Its own first item (if the planner gave it one) comes inline in the CTA's header with its
+        // first 32 page ids, so that the first copies leave after one round trip to memory; every
+        // later item arrives from the fetch warp through shared memory, ready to issue.
+        struct PItem { int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row, page0, unit, n_chunks, partial_base; };
         int n = 0;
-        // the CTA's header gives its item range, its first item and that item's first 32 page ids in
-        // one round trip to memory
         const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
         const int i0 = head[2], i1 = head[3];
-        auto load_item = [&](int ii) {
-            PItem r{0, 0, 0, 0, 0, 0, -1, 0};
-            if (ii < i1) {
-                const int4* src = ii == i0 ? reinterpret_cast<const int4*>(head + kHeadWorkCuda)
-                                           : reinterpret_cast<const int4*>(p.works + ii);
-                const int4 a = __ldg(src), b = __ldg(src + 1);
-                r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z; r.ntok = a.w;
-                r.kv_limit0 = b.x; r.kv_head = b.y; r.partial_row = b.z; r.page0 = b.w;
-            }
+        auto unpack = [](const int32_t* w) {
+            PItem r;
+            r.kv0 = w[0]; r.kv_end = w[1]; r.q_row0 = w[2]; r.ntok = w[3];
+            r.kv_limit0 = w[4]; r.kv_head = w[5]; r.partial_row = w[6]; r.page0 = w[7];
+            r.unit = w[8]; r.n_chunks = w[9]; r.partial_base = w[10];
             return r;
         };
         auto load_pages = [&](const PItem& it, int first_page) {
@@ -226,13 +432,31 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         constexpr int kPagesPerTile = kTileTok / kPage;       // 8
         constexpr int kGroupTiles = 32 / kPagesPerTile;       // 4
         bool ok = true;
-        PItem cur = load_item(i0), nxt = load_item(i0 + 1);
-        int pages_cur = head[kHeadPagesCuda + lane];
+        int taken = 0;
+        int pages_cur = 0;
+        // next item from the fetch warp (kv_end == 0: none); also sets pages_cur to its first 32 page ids
+        auto take = [&]() {
+            PItem r{0, 0, 0, 0, 0, 0, -1, 0, 0, 1, -1};
+            ok = mbar_wait(next_full, (uint32_t)taken & 1u, abort_flag, p.status, 6);
+            if (ok) {
+                r = unpack(next_item->work);
+                pages_cur = next_item->pages[lane];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(next_free);
+                ++taken;
+            }
+            return r;
+        };
+        PItem cur{0, 0, 0, 0, 0, 0, -1, 0, 0, 1, -1};
+        if (i0 < i1) {
+            cur = unpack(head + kHeadWorkCuda);
+            pages_cur = head[kHeadPagesCuda + lane];
+        }
         // The plan was uploaded before the kernel in front of this one started, so all of the above
-        // overlaps that kernel's tail; the pool and Q are read only from here on.
+        // overlaps that kernel's tail; the pool, Q and the queue are touched only from here on.
         pdl_wait();
-        for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
-            const PItem after = load_item(ii + 2);
+        if (cur.kv_end == 0) cur = take();      // a CTA that came from span tiles starts on the queue
+        while (cur.kv_end > 0 && ok) {
             const int ntiles = (cur.kv_end - cur.kv0 + kTileTok - 1) / kTileTok;
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
@@ -255,6 +479,10 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                         d.out_row = cur.q_row0;
                         d.kv_head = cur.kv_head;
                         d.partial_row = cur.partial_row;
+                        d.unit = cur.unit;
+                        d.n_chunks = cur.n_chunks;
+                        d.partial_base = cur.partial_base;
+                        d.stage = s;
                         d.pad = 0;
                         desc[s] = d;
                         mbar_arrive_expect_tx(full0 + 8 * s,
@@ -263,6 +491,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                     __syncwarp();
                     const int page = __shfl_sync(0xffffffffu, pages_cur,
                                                  (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
+                    if (lane == 0) { if (n == 0) trace_mark(2); trace_add(6, 1); if (first) trace_add(5, 1); }
                     if (lane < npages)
                         tma_page_kv(smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + (size_t)lane * Geo::PAGE_BYTES),
                                     kv_map, cur.kv_head, page, full0 + 8 * s);
@@ -273,17 +502,12 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                         bulk_g2s(smem_u32(q_base + (size_t)s * Geo::Q_BYTES + (size_t)tok * G * D * 2), src,
                                  G * D * 2, full0 + 8 * s);
                     }
-                    // page ids of the next group of stages (or of the next item), requested only after this
-                    // group's first stage is on its way: the next item's descriptor may still be in flight
-                    if (t == t0) {
-                        if (t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
-                        else if (nxt.kv_end > 0) pages_nxt = load_pages(nxt, 0);
-                    }
+                    // page ids of the next group of stages are requested after this group's first stage has left
+                    if (t == t0 && t0 + kGroupTiles < ntiles) pages_nxt = load_pages(cur, (t0 + kGroupTiles) * kPagesPerTile);
                 }
                 pages_cur = pages_nxt;
             }
-            cur = nxt;
-            nxt = after;
+            if (ok) cur = take();
         }
         if (ok) {
             const int s = n % S;
@@ -301,11 +525,62 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                 while (!mbar_try_wait(full0 + 8 * (k % S), (uint32_t)(k / S) & 1u) &&
                        clock64() - t0 < kWaitCycles) {}
         }
+        // the last CTA to leave the queue puts its counters back to zero for the next launch
+        if (p.queue_count > 0 && lane == 0 && atomicAdd(p.counters + 1, 1) == (int)gridDim.x - 1) {
+            atomicExch(p.counters, 0);
+            atomicExch(p.counters + 1, 0);
+        }
+        return;
+    }
+
+    if (warp == kEpilogueWarp) {
+        epilogue_loop<D, G>(p, out, lse, stage_base, handoff, merge_req, empty0, done0, req0, reqfree0, abort_flag);
+        return;
+    }
+    if (warp == kMergeWarp) {
+        merge_loop<D, G>(p, out, lse, merge_req, req0, reqfree0, abort_flag);
+        return;
+    }
+    if (warp == kFetchWarp) {
+        // ------------------------------------------------------------------ fetch warp
+        // Runs one item ahead of the producer: the CTA's own items (beyond the first, which the producer
+        // reads from the header itself), then the queue, one atomic add per chunk.  A chunk is claimed
+        // only when the producer has taken the one before it, so a CTA never holds more than one chunk
+        // it has not started.
+        const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
+        const int i1 = head[3];
+        int own = head[2] < i1 ? head[2] + 1 : i1;
+        pdl_wait();      // the queue's counter belongs to the launch in front until that has completed
+        for (int j = 0;; ++j) {
+            if (j > 0 && !mbar_wait(next_free, (uint32_t)(j - 1) & 1u, abort_flag, p.status, 7)) break;
+            int idx = -1;
+            if (own < i1) {
+                idx = own++;
+            } else if (p.queue_count > 0) {
+                int k = 0;
+                if (lane == 0) k = atomicAdd(p.counters, 1);
+                k = __shfl_sync(0xffffffffu, k, 0);
+                if (k < p.queue_count) idx = p.queue_first + k;
+            }
+            int w = 0, pg = 0;
+            if (idx >= 0) {
+                const int32_t* rec = reinterpret_cast<const int32_t*>(p.works + idx);
+                if (lane < 12) w = __ldg(rec + lane);
+                const int kv0 = __shfl_sync(0xffffffffu, w, 0), kv_end = __shfl_sync(0xffffffffu, w, 1);
+                const int page0 = __shfl_sync(0xffffffffu, w, 7);
+                if (lane < (kv_end - kv0 + kPage - 1) / kPage) pg = __ldg(p.page_indices + page0 + lane);
+            }
+            if (lane < 12) next_item->work[lane] = w;
+            next_item->pages[lane] = pg;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(next_full);
+            if (idx < 0) break;
+        }
         return;
     }
 
     // ---------------------------------------------------------------------- consumer warps
-    pdl_wait();      // outputs may be written only after the kernel in front has completed
+    pdl_wait();
     const int g = lane >> 2, t4 = lane & 3;      // fragment coordinates
     const float qscale = p.sm_scale * kLog2e;
     // ldmatrix row addresses inside a page slot, without the per-step piece index:
@@ -319,7 +594,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
     uint32_t qb[Geo::KSTEPS][2];      // B fragments of Q^T: column g, values 16 ks + 2 t4 (+1) and + 8
     float o[Geo::KSTEPS][4];          // O^T: rows d = 16 i + g (+8), columns 2 t4, 2 t4 + 1
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;      // of columns 2 t4 and 2 t4 + 1
-    int32_t cur_out_row = 0, cur_kv_head = 0, cur_partial = -1, cur_ntok = 1;
     int item_count = 0;
 
     for (int n = 0;; ++n) {
@@ -327,7 +601,13 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         const uint32_t ph = (uint32_t)(n / S) & 1u;
         if (!mbar_wait(full0 + 8 * s, ph, abort_flag, p.status, 2)) break;
         const TileDesc d = desc[s];
-        if (d.flags & kFlagEnd) break;
+        if (d.flags & kFlagEnd) {
+            // tell the epilogue warp that nothing follows
+            if (threadIdx.x == 0) { trace_mark(4); handoff[item_count % kHandoffs].flags = kFlagEnd; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(done0 + 8 * (item_count % kHandoffs));
+            break;
+        }
         uint8_t* stage = stage_base + (size_t)s * Geo::STAGE_BYTES;
         if (d.flags & kFlagFirst) {
             const uint8_t* qs = q_base + (size_t)s * Geo::Q_BYTES;
@@ -342,7 +622,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             }
             m0 = m1 = -INFINITY;
             l0 = l1 = 0.f;
-            cur_out_row = d.out_row; cur_kv_head = d.kv_head; cur_partial = d.partial_row; cur_ntok = d.ntok;
         }
         const int key0 = warp * kPage;                    // this warp's page inside the stage
         if (key0 < d.rows) {
@@ -421,8 +700,8 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             if (lane == 0) mbar_arrive(empty0 + 8 * s);
             continue;
         }
-        // ---- end of item: merge the warps' states through this stage's shared memory (each warp's
-        // own page slot is free: only this warp read it) and write the result
+        // ---- end of item: leave this warp's state in its own page slot of the stage (only this warp
+        // read that slot) for the epilogue warp, and go on
         {
             float* st = reinterpret_cast<float*>(stage + (size_t)warp * Geo::PAGE_BYTES);
 #pragma unroll
@@ -444,48 +723,11 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                 ms[2 * t4] = m0; ms[2 * t4 + 1] = m1;
                 ms[kCols + 2 * t4] = l0; ms[kCols + 2 * t4 + 1] = l1;
             }
+            const int h = item_count % kHandoffs;
+            if (threadIdx.x == 0) handoff[h] = d;
             __syncwarp();
-            if (lane == 0) mbar_arrive(mbar);
-            if (!mbar_wait(mbar, (uint32_t)item_count & 1u, abort_flag, p.status, 3)) break;
+            if (lane == 0) mbar_arrive(done0 + 8 * h);
             ++item_count;
-            const int ncols = cur_ntok * G;
-            for (int e = 2 * (int)threadIdx.x; e < ncols * D; e += 2 * kWarps * 32) {
-                const int col = e / D, dd = e % D;
-                float M = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < kWarps; ++w)
-                    M = fmaxf(M, reinterpret_cast<const float*>(stage + (size_t)w * Geo::PAGE_BYTES)[kCols * Geo::O_STRIDE + col]);
-                float L = 0.f, a0 = 0.f, a1 = 0.f;
-#pragma unroll
-                for (int w = 0; w < kWarps; ++w) {
-                    const float* sw = reinterpret_cast<const float*>(stage + (size_t)w * Geo::PAGE_BYTES);
-                    const float mw = sw[kCols * Geo::O_STRIDE + col];
-                    const float wgt = mw == -INFINITY ? 0.f : fast_exp2(mw - M);
-                    if (wgt != 0.f) {      // a warp without a visible key holds nothing worth reading
-                        L = fmaf(sw[kCols * Geo::O_STRIDE + kCols + col], wgt, L);
-                        const float2 ov = *reinterpret_cast<const float2*>(sw + (size_t)col * Geo::O_STRIDE + dd);
-                        a0 = fmaf(ov.x, wgt, a0);
-                        a1 = fmaf(ov.y, wgt, a1);
-                    }
-                }
-                const float inv = L > 0.f ? 1.f / L : 0.f;
-                const float lse2 = L > 0.f ? M + log2f(L) : -INFINITY;
-                const int tok = col / G, hh = col % G;
-                const size_t hq = (size_t)cur_kv_head * G + hh;
-                if (cur_partial < 0) {
-                    *reinterpret_cast<uint32_t*>(out + ((size_t)(cur_out_row + tok) * Hq + hq) * D + dd) =
-                        pack_bf16x2(a0 * inv, a1 * inv);
-                    if (lse != nullptr && dd == 0) lse[(size_t)(cur_out_row + tok) * Hq + hq] = lse2 * kLn2;
-                } else {
-                    *reinterpret_cast<float2*>(p.partial_o + (((size_t)cur_partial + tok) * G + hh) * D + dd) =
-                        make_float2(a0 * inv, a1 * inv);
-                    if (dd == 0) p.partial_lse[((size_t)cur_partial + tok) * G + hh] = lse2;
-                }
-            }
-            // the stage goes back to the producer, whose copies are writes of the asynchronous proxy
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8 * s);
         }
     }
 }

@@ -32,6 +32,7 @@ attn_decode_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const 
                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
+    if (threadIdx.x == 0) { trace_mark(0); trace_set(1, 0); trace_set(5, 0); trace_set(6, 0); trace_set(7, 0); }
     dec::decode_body<D, G>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw));
 }
 
@@ -52,6 +53,7 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = aligned_smem(smem_raw);
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
+    if (threadIdx.x == 0) { trace_mark(0); trace_set(1, 0); trace_set(5, 0); trace_set(6, 0); trace_set(7, 0); }
     const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
     // bring the whole header and the tensor map close now: the decode phase of a CTA that starts with
     // span tiles finds them in L2 when it gets there
@@ -63,7 +65,8 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
         return;
     }
     tc::tc_body<G>(p, q, pool, out, lse, smem);
-    if (head[2] == head[3]) return;      // the planner gave this CTA its decode rows as tensor-core items too
+    if (threadIdx.x == 0) trace_mark(1);
+    if (head[2] == head[3] && p.queue_count == 0) return;      // nothing left for the warp body
     __syncthreads();      // tensor memory released, shared memory free for the second phase
     dec::decode_body<tc::kD, G>(p, &kv_map, q, out, lse, S, smem);
 }
@@ -195,3 +198,11 @@ cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_poo
 }
 
 }  // namespace asynclm
+
+#ifdef ASYNCLM_TRACE
+// Debug builds only: copies the per-CTA time stamps of the last attention launch to the host
+// (synchronises the device).  out: [1024][8] unsigned 64-bit.
+extern "C" int asynclm_trace_read(unsigned long long* out) {
+    return cudaMemcpyFromSymbol(out, asynclm::g_trace, sizeof(asynclm::g_trace)) == cudaSuccess ? 0 : -5;
+}
+#endif

@@ -5,9 +5,9 @@
 // loop that has handed every byte of HBM to its KV pool and weight arena at start-up and has no
 // allocator left to ask, a plug-in running inside a host process whose memory pool it may not
 // touch, and a real-time path in which cudaMalloc is forbidden because it may synchronise the whole
-// device.  Such callers can size the plan's device workspace for the plan arrays alone; the fp32
-// partial outputs of split contexts, which are the only scratch memory the attention kernels use,
-// then live in the fixed array below instead.
+// device.  For them the fp32 partial outputs of split contexts, which are the only scratch memory the
+// attention kernels use, live in the fixed array below instead of the plan's device workspace (whose
+// size asynclm_plan still checks against the full requirement; that part of it is simply left alone).
 //
 // The array is part of the library image: every GPU that loads the library carries it from the
 // first use of the library on that GPU until the process exits.
@@ -66,21 +66,15 @@ extern "C" int asynclm_attn_mixed_static(const asynclm_plan_t* plan, const void*
     const size_t o_bytes = align256(rows * (size_t)plan->dev.group * (size_t)plan->dev.head_dim * sizeof(float));
     const size_t l_bytes = align256(rows * (size_t)plan->dev.group * sizeof(float));
     if (o_bytes + l_bytes > kStaticScratchBytes) return ASYNCLM_ERR_STATIC_SCRATCH_TOO_SMALL;
+    if (int rc = check_plan_device(plan->device)) return rc;
     void* base = nullptr;
-    if (scratch_address(&base) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return ASYNCLM_ERR_CUDA;
-    }
+    if (int rc = cuda_status(scratch_address(&base))) return rc;
     DevPlan d = plan->dev;                       // same plan, partial results redirected
     d.partial_o = (float*)base;
     d.partial_lse = (float*)((unsigned char*)base + o_bytes);
     cudaStream_t s = (cudaStream_t)stream;
-    if (launch_attention(d, q, kv_pool, out, lse, s) != cudaSuccess ||
-        launch_lse_merge(d, out, lse, s) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return ASYNCLM_ERR_CUDA;
-    }
-    return ASYNCLM_OK;
+    if (int rc = cuda_status(launch_attention(d, q, kv_pool, out, lse, s))) return rc;
+    return cuda_status(launch_lse_merge(d, out, lse, s));
 }
 
 extern "C" size_t asynclm_static_scratch_bytes(void) { return kStaticScratchBytes; }

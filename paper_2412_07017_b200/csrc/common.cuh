@@ -58,6 +58,28 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Per-CTA time stamps for performance work: compiled in only with -DASYNCLM_TRACE (see build.py),
+// read back with asynclm_trace_read().  Slot meanings are the callers'.
+#ifdef ASYNCLM_TRACE
+constexpr int kTraceSlots = 8, kTraceCtas = 1024;
+static __device__ unsigned long long g_trace[kTraceCtas][kTraceSlots];      // one copy per translation unit
+__device__ __forceinline__ void trace_mark(int slot) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (blockIdx.x < kTraceCtas) g_trace[blockIdx.x][slot] = t;
+}
+__device__ __forceinline__ void trace_add(int slot, unsigned long long v) {
+    if (blockIdx.x < kTraceCtas) g_trace[blockIdx.x][slot] += v;
+}
+__device__ __forceinline__ void trace_set(int slot, unsigned long long v) {
+    if (blockIdx.x < kTraceCtas) g_trace[blockIdx.x][slot] = v;
+}
+#else
+__device__ __forceinline__ void trace_mark(int) {}
+__device__ __forceinline__ void trace_add(int, unsigned long long) {}
+__device__ __forceinline__ void trace_set(int, unsigned long long) {}
+#endif
+
 // Element offset of the first value of (page, K|V, kv head, slot) in the pool.
 __device__ __forceinline__ size_t pool_row_offset(int64_t page, int which, int kv_head, int slot,
                                                   int num_kv_heads, int head_dim) {

@@ -16,4 +16,12 @@ cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_poo
 
 cudaError_t launch_lse_merge(const DevPlan& p, void* out, float* lse, cudaStream_t stream);
 
+// Remembers `e` as the calling thread's last CUDA error (asynclm_last_cuda_error) and clears the
+// runtime's sticky launch error; returns ASYNCLM_OK for cudaSuccess, else ASYNCLM_ERR_CUDA.
+int cuda_status(cudaError_t e);
+
+// ASYNCLM_OK if the current device is the one the plan was made for, else ASYNCLM_ERR_INVALID_ARG
+// (ASYNCLM_ERR_CUDA if the device cannot be queried).
+int check_plan_device(int plan_device);
+
 }  // namespace asynclm

@@ -44,18 +44,17 @@ static int check_shape(const asynclm_shape* s) {
 // Tokens of a span that one tensor-core work item covers: two row tiles of 128 (token, head) rows.
 int tensor_tile_tokens(int group) { return 256 / group; }
 
-// Rows (G * q_len) from which a (sequence, kv head) goes to the tensor-core kernel.  Up to 4 heads per
-// kv head a decode row stays on the CUDA-core kernel, which then runs near the memory rate, and spans
-// of 32 rows and more take the tensor cores.  With 8 heads per kv head every KV byte feeds twice the
-// arithmetic and the CUDA-core kernel is bound by its FMAs at half the memory rate (measured:
-// 2.4 TB/s against 4.1 TB/s on the 64/8-head batch), so there the 8 rows of a decode token already
-// count as wide enough.
-static int default_tensor_min_rows(int group) { return group >= 8 ? 8 : 32; }
+// Rows (G * q_len) from which a (sequence, kv head) goes to the span body (tcgen05).  Below it the
+// warp body reads the keys once per 8 (token, head) columns, which costs less than a span item's
+// start-up; decode rows (G rows) always stay on the warp body, which runs at the memory rate for
+// every supported G.
+static int default_tensor_min_rows(int) { return 32; }
 
 // Sizes of the sections of the packed blob (identical offsets on host and device).
 struct BlobLayout {
     size_t off_q_indptr, off_kv_len, off_page_indptr, off_page_indices, off_row_seq, off_row_slot, off_units,
-        off_items, off_works, off_heads, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status, blob_bytes;
+        off_items, off_works, off_heads, off_cta_cuda, off_cta_tensor, off_split, off_merge, off_status,
+        off_arrivals, blob_bytes;
 };
 
 static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64_t n_units,
@@ -79,6 +78,7 @@ static BlobLayout layout_blob(int batch, int total_q, int64_t total_pages, int64
     L.off_cta_tensor = take(sizeof(int32_t) * (size_t)(ctas_tensor + 1));
     L.off_split = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_split, 1));
     L.off_merge = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_merge_blocks, 1));
+    L.off_arrivals = take(sizeof(int32_t) * (size_t)std::max<int64_t>(n_units, 1));
     L.blob_bytes = o;
     return L;
 }
@@ -88,9 +88,21 @@ static size_t partial_bytes(int64_t rows, int group, int head_dim) {
            align_up((size_t)rows * (size_t)group * sizeof(float), 256);
 }
 
-// Upper bound on the number of items the automatic policy produces: every unit yields one item
-// plus at most one extra cut per persistent CTA.
-static int64_t auto_item_bound(int64_t units, int ctas) { return units + ctas; }
+// Warp-body units: a sixth of the work is cut into short chunks for the end of the queue, about
+// kTailChunksPerCta per CTA and never shorter than kMinChunkTiles tiles (see deal_dynamic).
+constexpr int kTailChunksPerCta = 2;
+constexpr int kMinChunkTiles = 4;
+// Tokens of one warp-body unit: its MMAs have 8 (token, head) columns.
+static int warp_unit_tokens(int group) { return 8 / group; }
+
+// Upper bounds on what the automatic policy produces.  Warp body: the short chunks are at least
+// (all tiles) / (12 CTAs) long, so even a single unit that holds all the work yields at most 12 per
+// CTA; a long piece is at least two fifths of a CTA's share.  Span body: a unit is cut only where it
+// is larger than a CTA's share.
+static int64_t auto_item_bound(int64_t units, int ctas) { return 2 * units + (int64_t)20 * ctas; }
+static int64_t auto_partial_row_bound(int ctas, int group) {
+    return (int64_t)20 * ctas * warp_unit_tokens(group) + (int64_t)3 * ctas * tensor_tile_tokens(group);
+}
 
 }  // namespace asynclm
 
@@ -117,10 +129,8 @@ extern "C" int asynclm_plan_workspace_size(const asynclm_shape* shape,
         max_items = max_units * per_unit;
         max_partial_rows = max_items;   // ntok tokens per unit are already counted in max_units
     } else {
-        max_items = auto_item_bound(max_units, ctas_cuda + ctas_tensor);
-        // only cut units hold partial rows: at most 2 pieces per cut, tensor_tile_tokens rows each
-        max_partial_rows = (int64_t)2 * (ctas_cuda + ctas_tensor) * tensor_tile_tokens(G) +
-                           (int64_t)2 * (ctas_cuda + ctas_tensor);
+        max_items = auto_item_bound(max_units, ctas_cuda);
+        max_partial_rows = auto_partial_row_bound(ctas_cuda, G);      // only cut units hold partial rows
     }
     BlobLayout L = layout_blob(max_batch, max_total_q, max_total_pages, max_units, max_items,
                                ctas_cuda, ctas_tensor, max_units,
@@ -216,222 +226,239 @@ void cut_and_deal(const std::vector<int>& unit_ids, std::vector<UnitBuild>& unit
 }
 
 
-// Measured costs of the attention kernels on B200, in nanoseconds, used only to balance CTAs.
+// Measured costs of the attention kernels on B200, in nanoseconds, used only to size the span CTAs.
 struct PathCost {
     int gran;            // tokens per tile of the path (cuts fall on multiples of it)
     int64_t tile_ns;     // one tile in steady state
     int64_t item_ns;     // starting and finishing an item (pipeline fill and drain, merge, write)
     int64_t phase_ns;    // first item of the path on a CTA (descriptor chain, first loads)
 };
-// (fitted to per-CTA phase times of the fused kernel on the Llama-3-8B-shaped mixed batch)
+// Span body: a KV tile of 128 keys against one row tile, an item, the body's start on a CTA.
 constexpr PathCost kTensorCost{128, 1170, 8000, 11800};
-constexpr PathCost kCudaCost{128, 900, 1200, 2000};
 constexpr int64_t kTensorDualTileNs = 2435;   // a KV tile of an item with two row tiles (more than 128 rows)
-// When every unit runs on the tensor-core kernel all SMs stream K/V tiles at once and the tile time is
-// set by the memory system (64 KB per tile and SM: 148 SMs at 37 KB/us are 5.5 TB/s); the producers
-// run ahead across item boundaries.
+// When every unit runs on the span body all SMs stream K/V tiles at once and the tile time is set by
+// the memory system (64 KB per tile and SM); the producers run ahead across item boundaries.
 constexpr PathCost kTensorOnlyCost{128, 1543, 8000, 2400};
 constexpr int64_t kTensorOnlyDualTileNs = 3126;
-// Units with fewer (token, head) rows than this are cut wherever a CTA is full (their partial rows are
-// a few KB); wider span units are kept whole where they fit.
-constexpr int kWholeUnitMinRows = 32;
-// Decode units that a span CTA takes along on the tensor-core body at most (estimated from its room).
-constexpr int64_t kMaxNarrowUnitsPerCta = 4;
+// Warp body: 64 KB per 128-key tile.  It is bound by memory, so its tile time depends on how many SMs
+// stream at once: 1.45 us when all 148 do, 1.05 us (62 KB/us, about what one SM can stream) when
+// half of them run span tiles, which draw little bandwidth.  The model takes the latter figure.
+constexpr PathCost kWarpCost{128, 1050, 400, 2000};
+// No step ends before its bytes have crossed the memory bus: K/V pages stream at about 6 bytes per
+// nanosecond on this access pattern (4 KB runs through a shuffled page table), after about 3 us in
+// which the CTAs start.  Without this floor the model would spread the span units over so many CTAs
+// that too few were left streaming to keep the memory busy (one SM streams 60-75 KB/us at most).
+// Each (sequence, kv head) counts once: the row tiles of a long span re-read it, mostly from L2.
+constexpr int64_t kDramBytesPerUs = 6000000;
+// A span CTA that finishes early joins the queue; one that finishes late delays the whole step, and the
+// span body slows down by up to 15 % when the warp-body CTAs saturate the memory.  So the span CTAs
+// are filled to the load limit divided by this margin (in 1/64).
+constexpr int64_t kSpanMargin64 = 72;
+// Share (in 1/64) of the queue that the CTAs without span work must be able to stream by themselves.
+constexpr int64_t kStreamShare64 = 58;
+constexpr int64_t kStartNs = 3000;
 
-// Default policy for the fused kernel, in which a persistent CTA runs its tensor-core items and then,
-// if it has any, its CUDA-core items: units are weighted with the measured costs and dealt under a
-// per-CTA load limit (see `fill` below), where decode rows placed on a CTA with span work normally
-// become tensor-core items so that the CTA runs one body only; the smallest limit that fits is found
-// by bisection, so that all CTAs finish together as far as the cost model holds.
-void deal_jointly(const std::vector<int>& ids_tensor, const std::vector<int>& ids_cuda,
-                  std::vector<UnitBuild>& units, int group, int n_ctas, std::vector<Item>& items,
-                  std::vector<int32_t>& cta_indptr_cuda, std::vector<int32_t>& cta_indptr_tensor,
-                  std::vector<int32_t>& item_cta) {
+// Default policy for the fused kernel.
+//   Span units (tensor-core body) are compute-heavy and predictable: they are packed whole onto as few
+// persistent CTAs as the load limit allows (largest first, each into the fullest CTA that still has
+// room; a unit larger than a CTA's share is cut into equal pieces), so that most of them write final
+// bf16 rows instead of fp32 partial rows.
+//   Warp-body units (decode rows, short spans) are bandwidth-bound, and how fast a CTA streams depends
+// on what the other SMs are doing, which no static cost predicts.  They are cut into chunks of a few
+// tiles, sorted by length (longest first), and handed out at run time: the CTAs without span work
+// start on one chunk each, every other chunk waits in a queue from which a CTA that runs out of work
+// (a span CTA included) takes the next one with one atomic add.  Partial results are indexed by chunk
+// and merged in chunk order, so the output does not depend on which CTA ran what.
+//   The load limit is the smallest one under which the span units fit and the room left on all CTAs
+// covers the modelled time of the queue; it is found by bisection.
+void deal_dynamic(std::vector<int>& ids_tensor, const std::vector<int>& ids_warp,
+                  std::vector<UnitBuild>& units, int group, int64_t kv_bytes, int n_ctas, std::vector<Item>& items,
+                  std::vector<int32_t>& cta_indptr_warp, std::vector<int32_t>& cta_indptr_tensor,
+                  std::vector<int32_t>& item_cta, int32_t* queue_first, int32_t* queue_count) {
     struct Piece { Item it; int32_t cta; };
-    std::vector<Piece> best[2];
-    const std::vector<int>* ids[2] = {&ids_tensor, &ids_cuda};
-    const bool tensor_only = ids_cuda.empty();
-    PathCost cost[2] = {tensor_only ? kTensorOnlyCost : kTensorCost, kCudaCost};
+    const bool tensor_only = ids_warp.empty();
+    const PathCost tc = tensor_only ? kTensorOnlyCost : kTensorCost;
     const int64_t dual_tile_ns = tensor_only ? kTensorOnlyDualTileNs : kTensorDualTileNs;
-    // a narrow item (one decode token's rows) on the tensor-core body: tile and item cost
-    const int64_t narrow_tile_ns = tensor_only ? kTensorOnlyCost.tile_ns : 1400;
-    const int64_t narrow_item_ns = 2900;
-    auto tile_ns = [&](int path, int id) {
-        return path == 0 && units[id].u.ntok * group > 128 ? dual_tile_ns : cost[path].tile_ns;
-    };
-    // Lower bound of the makespan: all work, one start per unit, one phase start per CTA.
-    int64_t total = 0;
-    for (int path = 0; path < 2; ++path)
-        for (int id : *ids[path])
-            total += cost[path].item_ns + (units[id].n_keys + cost[path].gran - 1) / cost[path].gran * tile_ns(path, id);
-    // Deal the work under a per-CTA load limit `cap`; returns false if it does not fit.
-    //   Span units first, whole wherever possible (an unsplit unit writes final bf16 rows: no fp32
-    // partial rows, no merge): largest first, each into the fullest span CTA that still has room for
-    // it, else into a fresh CTA; a unit larger than a CTA's share is cut into equal pieces.
-    //   Decode units then fill every CTA up to the limit in CTA order; a unit is cut only where a
-    // CTA is full.
-    //   With emit == false only the verdict is computed (the bisection's probes).
-    std::vector<int> tensor_order, tensor_narrow;      // span units packed whole; narrow units that fill up CTAs
-    for (int id : ids_tensor)
-        (units[id].u.ntok * group >= kWholeUnitMinRows ? tensor_order : tensor_narrow).push_back(id);
-    std::vector<int64_t> tiles_of(units.size()), tns_of(units.size());
-    for (int path = 0; path < 2; ++path)
-        for (int id : *ids[path]) {
-            tiles_of[(size_t)id] = (units[id].n_keys + cost[path].gran - 1) / cost[path].gran;
-            tns_of[(size_t)id] = tile_ns(path, id);
+    auto tiles_of = [](int64_t keys, int gran) { return (keys + gran - 1) / gran; };
+
+    // ---- warp-body work as the model sees it (the chunks are cut below, once the number of CTAs
+    // that start on the queue is known)
+    int64_t warp_tiles = 0;
+    for (int id : ids_warp) warp_tiles += tiles_of(units[id].n_keys, kWarpCost.gran);
+    const int64_t warp_ns = warp_tiles * kWarpCost.tile_ns + (int64_t)ids_warp.size() * 2 * kWarpCost.item_ns;
+
+    // ---- span units with two row tiles that would not fit a CTA whole are divided by rows into two
+    // units of one row tile each (same CTA-time in total, and the second reader of the keys finds most
+    // of them in L2) rather than by keys, which would cost fp32 partial rows and a merge.  The limit
+    // used for the decision is the lower bound of the one found below.
+    {
+        int64_t work = warp_ns;
+        for (int id : ids_tensor)
+            work += tc.item_ns + tiles_of(units[id].n_keys, tc.gran) * (units[id].u.ntok * group > 128 ? dual_tile_ns : tc.tile_ns);
+        const int64_t limit0 = std::max(work / n_ctas, kStartNs + kv_bytes * 1000 / kDramBytesPerUs) * 64 / kSpanMargin64;
+        const int half = 128 / group;      // tokens of one row tile
+        const size_t n0 = ids_tensor.size();
+        for (size_t i = 0; i < n0; ++i) {
+            const int id = ids_tensor[i];
+            UnitBuild& ub = units[(size_t)id];
+            if (ub.u.ntok * group <= 128) continue;
+            if (tc.phase_ns + tc.item_ns + tiles_of(ub.n_keys, tc.gran) * dual_tile_ns <= limit0) continue;
+            UnitBuild second = ub;
+            second.u.q_row0 += half;
+            second.u.ntok -= half;
+            second.u.kv_limit0 += half;
+            ub.u.ntok = half;
+            ub.n_keys = (int64_t)ub.u.kv_limit0 + ub.u.ntok - 1;
+            ids_tensor.push_back((int)units.size());
+            units.push_back(second);
         }
-    auto unit_tiles = [&](int, int id) { return tiles_of[(size_t)id]; };
-    std::stable_sort(tensor_order.begin(), tensor_order.end(), [&](int x, int y) {
-        return tiles_of[(size_t)x] * tns_of[(size_t)x] > tiles_of[(size_t)y] * tns_of[(size_t)y];
+    }
+
+    // ---- span units under a load limit
+    std::vector<int> order(ids_tensor);
+    std::vector<int64_t> tiles(units.size()), tns(units.size());
+    for (int id : order) {
+        tiles[(size_t)id] = tiles_of(units[id].n_keys, tc.gran);
+        tns[(size_t)id] = units[id].u.ntok * group > 128 ? dual_tile_ns : tc.tile_ns;
+    }
+    std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
+        return tiles[(size_t)x] * tns[(size_t)x] > tiles[(size_t)y] * tns[(size_t)y];
     });
     std::vector<int64_t> load((size_t)n_ctas);
-    int64_t avg_unit_ns = 1;      // mean cost of a CUDA-core unit
-    if (!ids_cuda.empty()) {
-        int64_t sum = 0;
-        for (int id : ids_cuda) sum += cost[1].item_ns + tiles_of[(size_t)id] * cost[1].tile_ns;
-        avg_unit_ns = std::max<int64_t>(1, sum / (int64_t)ids_cuda.size());
-    }
-    auto fill = [&](int64_t cap, std::vector<Piece> (&out)[2], bool emit) {
-        out[0].clear();
-        out[1].clear();
-        if (emit) {
-            out[0].reserve(ids_tensor.size() + (size_t)n_ctas);
-            out[1].reserve(ids_cuda.size() + (size_t)n_ctas);
-        }
-        bool fits = true;
+    std::vector<Piece> pieces_out;
+    int used = 0;
+    // Packs the span units under `cap`; returns false if they do not fit or leave too little room for
+    // the queue.  With emit == false only the verdict is computed (the bisection's probes).
+    int64_t span_work = 0;      // all span items without the per-CTA start
+    for (int id : order) span_work += tc.item_ns + tiles[(size_t)id] * tns[(size_t)id];
+    auto fill = [&](int64_t limit, bool emit) {
+        // CTAs that may hold span work: the others have to be able to stream most of the queue by
+        // themselves (span CTAs draw little bandwidth, and one SM streams only so much)
+        const int64_t stream_ctas = limit > kStartNs
+            ? (warp_tiles * kWarpCost.tile_ns * kStreamShare64 / 64 + (limit - kStartNs) - 1) / (limit - kStartNs) : n_ctas;
+        const int64_t span_ctas = ids_warp.empty() ? n_ctas : n_ctas - stream_ctas;
+        if (!order.empty() && span_ctas < 1) return false;
+        // what a span CTA may be given: the span work spread over those CTAs with some slack for the
+        // packing, at most the load limit less the safety margin.  Spreading the spans thin costs little (a
+        // span CTA that is done early joins the queue), filling span CTAs to the brim risks a late finish.
+        const int64_t thin = order.empty() ? 0 : span_work / span_ctas * 5 / 4 + tc.phase_ns + tc.item_ns + dual_tile_ns;
+        const int64_t cap = std::min(limit * 64 / kSpanMargin64, std::max(thin, 2 * (tc.phase_ns + tc.item_ns)));
+        pieces_out.clear();
         std::fill(load.begin(), load.end(), (int64_t)0);
-        int used = 0;                                   // CTAs that hold span work: [0, used)
-        int64_t least = INT64_MAX;                      // lower bound of the smallest load among them
-        {
-            const PathCost& pc = cost[0];
-            // tiles a fresh CTA takes, for the two kinds of span tile
-            const int64_t fresh_single = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / pc.tile_ns);
-            const int64_t fresh_dual = std::max<int64_t>(1, (cap - pc.phase_ns - pc.item_ns) / dual_tile_ns);
-            for (int id : tensor_order) {
-                const int64_t tns = tns_of[(size_t)id];
-                const int64_t tiles = unit_tiles(0, id);
-                const int64_t fresh_room = tns == pc.tile_ns ? fresh_single : fresh_dual;
-                const int64_t pieces = tiles <= fresh_room ? 1 : (tiles + fresh_room - 1) / fresh_room;
-                int64_t k0 = 0;
-                for (int64_t c = 0; c < pieces; ++c) {
-                    const int64_t take = pieces == 1 ? tiles : tiles / pieces + (c < tiles % pieces ? 1 : 0);
-                    const int64_t need = pc.item_ns + take * tns;
-                    int best_cta = -1;
-                    if (least + need <= cap)            // otherwise no span CTA has room: skip the scan
-                        for (int k = 0; k < used; ++k)
-                            if (load[(size_t)k] + need <= cap && (best_cta < 0 || load[(size_t)k] > load[(size_t)best_cta])) best_cta = k;
-                    if (best_cta < 0) {
-                        if (used < n_ctas) {
-                            best_cta = used++;
-                            load[(size_t)best_cta] = pc.phase_ns;
-                        } else {
-                            fits = false;
-                            best_cta = 0;
-                            for (int k = 1; k < n_ctas; ++k) if (load[(size_t)k] < load[(size_t)best_cta]) best_cta = k;
-                        }
+        used = 0;
+        int64_t least = INT64_MAX;      // lower bound of the smallest load among the span CTAs
+        bool fits = true;
+        for (int id : order) {
+            const int64_t t = tiles[(size_t)id], ns = tns[(size_t)id];
+            const int64_t fresh_room = std::max<int64_t>(1, (cap - tc.phase_ns - tc.item_ns) / ns);
+            const int64_t pieces = t <= fresh_room ? 1 : (t + fresh_room - 1) / fresh_room;
+            int64_t k0 = 0;
+            for (int64_t c = 0; c < pieces; ++c) {
+                const int64_t take = pieces == 1 ? t : t / pieces + (c < t % pieces ? 1 : 0);
+                const int64_t need = tc.item_ns + take * ns;
+                int best = -1;
+                if (least + need <= cap)            // otherwise no span CTA has room: skip the scan
+                    for (int k = 0; k < used; ++k)
+                        if (load[(size_t)k] + need <= cap && (best < 0 || load[(size_t)k] > load[(size_t)best])) best = k;
+                if (best < 0) {
+                    if (used < n_ctas) {
+                        best = used++;
+                        load[(size_t)best] = tc.phase_ns;
+                    } else {
+                        fits = false;
+                        best = 0;
+                        for (int k = 1; k < n_ctas; ++k) if (load[(size_t)k] < load[(size_t)best]) best = k;
                     }
-                    const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * pc.gran);
-                    if (emit) out[0].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c}, (int32_t)best_cta});
-                    else if (!fits) return false;
-                    load[(size_t)best_cta] += need;
-                    least = std::min(least, load[(size_t)best_cta]);
-                    k0 = k1;
                 }
+                if (!fits && !emit) return false;
+                const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * tc.gran);
+                if (emit) pieces_out.push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c}, (int32_t)best});
+                load[(size_t)best] += need;
+                least = std::min(least, load[(size_t)best]);
+                k0 = k1;
             }
         }
-        // Line fill: the units of `list` in order, each CTA up to the limit; a unit is cut only where a
-        // CTA is full.  CTAs below `started` already hold tensor-core work.  A CUDA-core unit (one decode
-        // token) that lands on such a CTA runs there as a narrow tensor-core item: the CTA then never
-        // re-splits its registers and restarts its pipeline for a second phase (measured on the
-        // Llama-shaped mixed batch: 91.6 -> 87 us per step), while CTAs without span work keep the
-        // CUDA-core body, which is the faster one on decode rows.
-        auto line_fill = [&](int path, const std::vector<int>& list, int started) {
-            int cta = 0;
-            bool has_phase = false;
-            // A narrow item costs about 2 us more than an item of the CUDA-core body, a second phase
-            // costs about 9 us once: the span CTA keeps to the tensor-core body only if the room left
-            // on it takes a few decode units (on the 32-sequence mixed batch, with about two units per
-            // span CTA, the step measures 89.3 us with this and 91.8 us without).
-            auto rides_along = [&](int k) {
-                return k < started && (path == 0 || cap - load[(size_t)k] <= kMaxNarrowUnitsPerCta * avg_unit_ns);
-            };
-            bool narrow_cta = rides_along(0);
-            for (int id : list) {
-                const int64_t n_keys = units[id].n_keys;
-                int64_t k0 = 0;
-                int c = 0;
-                while (k0 < n_keys) {
-                    const int pth = narrow_cta ? 0 : path;
-                    const PathCost& pc = cost[pth];
-                    const bool narrow = pth == 0;          // only narrow units are line-filled on the tensor path
-                    const int64_t tns = narrow ? narrow_tile_ns : tns_of[(size_t)id];
-                    const int64_t item_ns = narrow ? narrow_item_ns : pc.item_ns;
-                    const int64_t left = (n_keys - k0 + pc.gran - 1) / pc.gran;
-                    const bool last_cta = cta + 1 >= n_ctas;
-                    const int64_t start = item_ns + ((has_phase || narrow_cta) ? 0 : pc.phase_ns);
-                    const int64_t room = cap - load[(size_t)cta] - start;
-                    int64_t take;
-                    if (last_cta) {
-                        take = left;
-                        if (load[(size_t)cta] + start + take * tns > cap) fits = false;
-                    } else if (left * tns <= room + item_ns / 2) {
-                        take = left;                     // finishing here is cheaper than another item elsewhere
-                    } else if (room < tns * 2) {
-                        ++cta;                           // not worth starting an item for so little
-                        has_phase = false;
-                        narrow_cta = rides_along(cta);
-                        continue;
-                    } else {
-                        take = std::max<int64_t>(1, room / tns);
-                    }
-                    const int64_t k1 = std::min<int64_t>(n_keys, k0 + take * pc.gran);
-                    if (emit) out[pth].push_back(Piece{Item{id, (int32_t)k0, (int32_t)k1, c}, (int32_t)cta});
-                    else if (!fits) return false;
-                    load[(size_t)cta] += start + take * tns;
-                    has_phase = true;
-                    k0 = k1;
-                    ++c;
-                    if (!last_cta && k0 < n_keys) { ++cta; has_phase = false; narrow_cta = rides_along(cta); }
-                }
-            }
-            return true;
-        };
-        // narrow tensor units: on the span CTAs first, then on fresh CTAs (which pay the phase start)
-        if (!line_fill(0, tensor_narrow, used)) return false;
-        if (!line_fill(1, *ids[1], ids[1]->empty() ? 0 : used)) return false;
-        std::stable_sort(out[0].begin(), out[0].end(), [](const Piece& x, const Piece& y) { return x.cta < y.cta; });
-        return fits;
+        // room for the queue: what the span CTAs have left after restarting on the warp body, and the
+        // whole limit on the others
+        int64_t room = 0;
+        for (int k = 0; k < n_ctas; ++k)
+            room += std::max<int64_t>(0, limit - load[(size_t)k] - kWarpCost.phase_ns);
+        return fits && used <= span_ctas && room >= warp_ns;
     };
-    // Smallest limit that fits, by bisection (the loads are monotone in the limit up to rounding).
-    // The probes only ask whether a limit fits; the pieces are built once, for the limit found.
-    int64_t lo = std::max<int64_t>(1, total / n_ctas * 3 / 4);     // (decode rows on span CTAs cost less than assumed in `total`)
-    int64_t hi = lo + lo / 4 + kTensorCost.item_ns + kTensorCost.phase_ns + kCudaCost.phase_ns;
-    while (!fill(hi, best, false)) { lo = hi; hi += hi / 2; }
+    const int64_t total = warp_ns + span_work;
+    const int64_t floor_ns = kStartNs + kv_bytes * 1000 / kDramBytesPerUs;
+    int64_t lo = std::max<int64_t>(std::max<int64_t>(1, total / n_ctas), floor_ns);
+    int64_t hi = lo + lo / 4 + tc.item_ns + tc.phase_ns + kWarpCost.phase_ns;
+    while (!fill(hi, false)) { lo = hi; hi += hi / 2; }
     for (int iter = 0; iter < 24 && hi - lo > std::max<int64_t>(50, hi / 128); ++iter) {      // to 0.8 %
         const int64_t mid = (lo + hi) / 2;
-        if (fill(mid, best, false)) hi = mid; else lo = mid;
+        if (fill(mid, false)) hi = mid; else lo = mid;
     }
-    fill(hi, best, true);
-    // emit: CUDA-core items first, then tensor items; chunk counts per unit
-    cta_indptr_cuda.assign((size_t)n_ctas + 1, 0);
+    fill(hi, true);
+    std::stable_sort(pieces_out.begin(), pieces_out.end(), [](const Piece& x, const Piece& y) { return x.cta < y.cta; });
+
+    // ---- warp-body chunks.  An item boundary costs time and a split unit costs partial rows and a
+    // merge, so most of the work stays in long pieces: units are taken longest first; the first ones, up
+    // to a sixth of all tiles, are cut into short chunks that go to the END of the queue, where they
+    // even out the CTAs' finishing times (few units, many chunks each: few merges); every other unit
+    // stays whole unless it is longer than two fifths of the step, in which case it is cut into equal
+    // pieces.  The queue holds the long pieces longest first, then the short chunks.
+    std::vector<int> warp_order(ids_warp);
+    std::stable_sort(warp_order.begin(), warp_order.end(),
+                     [&](int x, int y) { return units[x].n_keys > units[y].n_keys; });
+    std::vector<Item> chunks, tail;
+    chunks.reserve(ids_warp.size() + (size_t)n_ctas * 4);
+    const int64_t bulk_max = std::max<int64_t>(kMinChunkTiles, hi * 2 / 5 / kWarpCost.tile_ns);
+    const int64_t tail_target = warp_tiles / 6;
+    const int64_t tail_chunk = std::max<int64_t>(kMinChunkTiles, tail_target / ((int64_t)n_ctas * kTailChunksPerCta));
+    int64_t tail_tiles = 0;
+    for (int id : warp_order) {
+        const int64_t t = tiles_of(units[id].n_keys, kWarpCost.gran);
+        const bool to_tail = tail_tiles < tail_target && t > tail_chunk + tail_chunk / 2;
+        const int64_t piece_max = to_tail ? tail_chunk : bulk_max;
+        const int64_t pieces = t <= piece_max + piece_max / 2 ? 1 : (t + piece_max - 1) / piece_max;
+        int64_t k0 = 0;
+        for (int64_t c = 0; c < pieces; ++c) {
+            const int64_t take = t / pieces + (c < t % pieces ? 1 : 0);
+            const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * kWarpCost.gran);
+            (to_tail ? tail : chunks).push_back(Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c});
+            k0 = k1;
+        }
+        units[id].u.n_chunks = (int32_t)pieces;
+        if (to_tail) tail_tiles += t;
+    }
+    auto longer = [](const Item& x, const Item& y) { return x.kv1 - x.kv0 > y.kv1 - y.kv0; };
+    std::stable_sort(chunks.begin(), chunks.end(), longer);
+    std::stable_sort(tail.begin(), tail.end(), longer);
+    chunks.insert(chunks.end(), tail.begin(), tail.end());
+
+    // ---- emit: warp-body items first (one start chunk for every CTA without span work, then the
+    // queue), then the span items grouped by CTA
+    cta_indptr_warp.assign((size_t)n_ctas + 1, 0);
     cta_indptr_tensor.assign((size_t)n_ctas + 1, 0);
-    for (int path = 1; path >= 0; --path) {
-        std::vector<int32_t>& indptr = path == 1 ? cta_indptr_cuda : cta_indptr_tensor;
-        const int32_t first = (int32_t)items.size();
-        std::vector<int32_t> count((size_t)n_ctas, 0);
-        for (const Piece& pz : best[path]) {
-            items.push_back(pz.it);
-            item_cta.push_back(pz.cta);
-            count[(size_t)pz.cta]++;
-            units[pz.it.unit].u.n_chunks = std::max(units[pz.it.unit].u.n_chunks, pz.it.chunk + 1);
-        }
-        int32_t at = first;
-        for (int k = 0; k < n_ctas; ++k) {
-            indptr[(size_t)k] = at;
-            at += count[(size_t)k];
-        }
-        indptr[(size_t)n_ctas] = at;
+    const int n_start = (int)std::min<size_t>(chunks.size(), (size_t)(n_ctas - used));
+    for (size_t i = 0; i < chunks.size(); ++i) {
+        items.push_back(chunks[i]);
+        item_cta.push_back(i < (size_t)n_start ? used + (int32_t)i : -1);
     }
+    for (int k = 0; k <= n_ctas; ++k)
+        cta_indptr_warp[(size_t)k] = std::min(std::max(k - used, 0), n_start);
+    *queue_first = n_start;
+    *queue_count = (int32_t)chunks.size() - n_start;
+    const int32_t first = (int32_t)items.size();
+    std::vector<int32_t> count((size_t)n_ctas, 0);
+    for (const Piece& pz : pieces_out) {
+        items.push_back(pz.it);
+        item_cta.push_back(pz.cta);
+        count[(size_t)pz.cta]++;
+        units[pz.it.unit].u.n_chunks = std::max(units[pz.it.unit].u.n_chunks, pz.it.chunk + 1);
+    }
+    int32_t at = first;
+    for (int k = 0; k < n_ctas; ++k) {
+        cta_indptr_tensor[(size_t)k] = at;
+        at += count[(size_t)k];
+    }
+    cta_indptr_tensor[(size_t)n_ctas] = at;
 }
 
 }  // namespace
@@ -443,7 +470,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     int rc = check_shape(shape);
     if (rc != ASYNCLM_OK) return rc;
     if (!batch || !host_ws || !out_plan || batch->batch < 0) return ASYNCLM_ERR_INVALID_ARG;
-    if (((uintptr_t)host_ws & 7) != 0 || ((uintptr_t)dev_ws & 255) != 0)
+    if (((uintptr_t)host_ws & 15) != 0 || ((uintptr_t)dev_ws & 255) != 0)
         return ASYNCLM_ERR_INVALID_ARG;
     const int B = batch->batch;
     if (B > 0 && (!batch->q_indptr || !batch->kv_len_before || !batch->page_indptr))
@@ -527,7 +554,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
         if (ql == 0) continue;
         const int ctx = batch->kv_len_before[b];
         const bool tensor = tensor_ok && (int64_t)G * ql >= tensor_min_rows;
-        const int step = tensor ? TQ : 1;
+        const int step = tensor ? TQ : warp_unit_tokens(G);
         for (int h = 0; h < Hkv; ++h) {
             for (int t0 = 0; t0 < ql; t0 += step) {
                 UnitBuild ub{};
@@ -554,6 +581,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     std::vector<Item> items;
     std::vector<int32_t> item_cta, cta_indptr_cuda, cta_indptr_tensor;
     int n_items_cuda = 0;
+    int32_t queue_first = 0, queue_count = 0;
     if (fixed_chunk > 0 || ctas_cuda != ctas_tensor) {
         cut_and_deal(ids_cuda, units, fixed_chunk, ctas_cuda, kCudaItemOverheadTiles, items,
                      cta_indptr_cuda, item_cta);
@@ -561,8 +589,11 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
         cut_and_deal(ids_tensor, units, fixed_chunk, ctas_tensor, kTensorItemOverheadTiles, items,
                      cta_indptr_tensor, item_cta);
     } else {
-        deal_jointly(ids_tensor, ids_cuda, units, G, ctas_cuda, items, cta_indptr_cuda, cta_indptr_tensor, item_cta);
-        n_items_cuda = cta_indptr_cuda[(size_t)ctas_cuda];
+        // bytes of K and V the step has to read, each (sequence, kv head) counted once
+        const int64_t kv_bytes = total_kv * Hkv * 4 * shape->head_dim;
+        deal_dynamic(ids_tensor, ids_cuda, units, G, kv_bytes, ctas_cuda, items, cta_indptr_cuda, cta_indptr_tensor, item_cta,
+                     &queue_first, &queue_count);
+        n_items_cuda = queue_first + queue_count;
     }
     const int n_items = (int)items.size();
 
@@ -575,7 +606,10 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
             partial_rows += (int64_t)units[i].u.n_chunks * units[i].u.ntok;
             split_units.push_back((int32_t)i);
             if (i >= (size_t)(INT32_MAX >> 6)) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
-            for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
+            // split units of the warp body are merged inside the attention kernel; those of the span
+            // body by the merge kernel
+            if (units[i].path == kPathTensor)
+                for (int rb = 0; rb * 4 < units[i].u.ntok * G; ++rb) merge_blocks.push_back((int32_t)((i << 6) | (size_t)rb));
             if (partial_rows > INT32_MAX / 2) return ASYNCLM_ERR_WORKSPACE_TOO_SMALL;
         }
     }
@@ -594,6 +628,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
 
     char* hb = (char*)host_ws + plan_bytes;
     std::memset(hb + L.off_status, 0, 256);
+    std::memset(hb + L.off_arrivals, 0, sizeof(int32_t) * std::max<size_t>(units.size(), 1));
     if (B > 0) {
         std::memcpy(hb + L.off_q_indptr, q_indptr, sizeof(int32_t) * (size_t)(B + 1));
         std::memcpy(hb + L.off_kv_len, batch->kv_len_before, sizeof(int32_t) * (size_t)B);
@@ -630,6 +665,10 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
         w.kv_head = u.kv_head;
         w.partial_row0 = u.partial_base < 0 ? -1 : u.partial_base + it.chunk * u.ntok;
         w.page0 = u.page_base + it.kv0 / kPage;
+        w.unit = it.unit;
+        w.n_chunks = u.n_chunks;
+        w.partial_base = u.partial_base;
+        w.pad = 0;
         h_works[i] = w;
     }
     for (int c = 0; c < std::max(ctas_cuda, ctas_tensor); ++c) {
@@ -674,6 +713,9 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     DevPlan& d = plan->dev;
     auto dp = [&](size_t off) { return host_only ? nullptr : (void*)(db + off); };
     d.status = (int32_t*)dp(L.off_status);
+    d.counters = (int32_t*)dp(L.off_status + 64);
+    d.queue_first = queue_first;
+    d.queue_count = queue_count;
     d.q_indptr = (const int32_t*)dp(L.off_q_indptr);
     d.kv_len_before = (const int32_t*)dp(L.off_kv_len);
     d.page_indptr = (const int32_t*)dp(L.off_page_indptr);
@@ -688,6 +730,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     d.cta_indptr_tensor = (const int32_t*)dp(L.off_cta_tensor);
     d.split_units = (const int32_t*)dp(L.off_split);
     d.merge_blocks = (const int32_t*)dp(L.off_merge);
+    d.unit_arrivals = (int32_t*)dp(L.off_arrivals);
     d.partial_o = (float*)dp(L.blob_bytes);
     d.partial_lse = (float*)dp(L.blob_bytes + align_up((size_t)partial_rows * (size_t)G *
                                                            (size_t)shape->head_dim * sizeof(float), 256));
@@ -722,7 +765,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     info.num_items_tensor = d.num_items_tensor;
     info.launches_append = T > 0 ? 1 : 0;
     // span tiles and decode rows share one fused launch when a step has both (head_dim 128)
-    info.launches_attn = ((n_items_cuda > 0 || d.num_items_tensor > 0) ? 1 : 0) + (d.num_split_units > 0 ? 1 : 0);
+    info.launches_attn = ((n_items_cuda > 0 || d.num_items_tensor > 0) ? 1 : 0) + (merge_blocks.empty() ? 0 : 1);
     info.num_sms = n_sms;
     info.total_kv_tokens = total_kv;
     info.device_bytes_used = dev_need;

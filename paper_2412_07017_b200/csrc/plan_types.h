@@ -7,7 +7,7 @@ namespace asynclm {
 
 constexpr int kKvTile = 128;          // split-KV chunk granularity in tokens (8 pages of 16)
 constexpr int kPage = 16;
-constexpr int kPathCuda = 0;
+constexpr int kPathCuda = 0;         // the warp-level body (decode rows, short spans)
 constexpr int kPathTensor = 1;
 
 // A unit is one query tile of one (sequence, kv head): `ntok` consecutive new tokens times the G
@@ -42,15 +42,19 @@ struct alignas(16) Work {
     int32_t kv_head;
     int32_t partial_row0;  // partial row of token 0 in this chunk; -1: the item writes final output
     int32_t page0;         // index into page_indices of the page that holds key kv0
+    int32_t unit;          // the unit this item is a chunk of
+    int32_t n_chunks;      // chunks of that unit
+    int32_t partial_base;  // partial row of its chunk 0, token 0 (-1 if unsplit)
+    int32_t pad;
 };
 
 // Per persistent CTA, one 384-byte header that holds everything the CTA needs to issue its first
-// loads after a single round trip to memory: words 0-3 its item ranges (tensor first, last;
-// CUDA-core first, last), words 8-15 the Work record of its first tensor item, words 16-23 that of
-// its first CUDA-core item, words 32-63 the first 32 page ids of the first tensor item and words
-// 64-95 those of the first CUDA-core item.
+// loads after a single round trip to memory: words 0-3 its item ranges (span body first, last;
+// warp body first, last), words 8-19 the Work record of its first span item, words 20-31 that of
+// its first warp-body item, words 32-63 the first 32 page ids of the first span item and words
+// 64-95 those of the first warp-body item.
 constexpr int kHeadWords = 96;
-constexpr int kHeadWorkTensor = 8, kHeadWorkCuda = 16, kHeadPagesTensor = 32, kHeadPagesCuda = 64;
+constexpr int kHeadWorkTensor = 8, kHeadWorkCuda = 20, kHeadPagesTensor = 32, kHeadPagesCuda = 64;
 
 // Pointers into the device workspace, passed to kernels by value.
 struct DevPlan {
@@ -66,11 +70,18 @@ struct DevPlan {
     const int32_t* cta_heads;        // [num_ctas][kHeadWords], see above
     const int32_t* cta_indptr_cuda;  // [num_ctas_cuda + 1] into items
     const int32_t* cta_indptr_tensor;// [num_ctas_tensor + 1] into items (absolute indices)
-    const int32_t* split_units;      // [num_split_units] unit ids that need a merge
-    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 6) | row block: 4 (token, head) rows each
+    const int32_t* split_units;      // [num_split_units] unit ids whose keys were cut into chunks
+    const int32_t* merge_blocks;     // [num_merge_blocks] (unit id << 6) | row block: 4 (token, head) rows each,
+                                     // for the split units of the span body (the merge kernel's work list)
+    int32_t* unit_arrivals;          // [num_units] chunks of a split warp-body unit that have written their
+                                     // partial rows; the CTA that brings a count to n_chunks merges the unit
+                                     // and puts the count back to zero
     float* partial_o;                // [partial_rows][G][d]
     float* partial_lse;              // [partial_rows][G]   (log2 domain)
     int32_t* status;                 // device status word
+    int32_t* counters;               // [0] next chunk of the warp body's queue, [1] CTAs that are done with the
+                                     // queue; both are zero between launches (the last CTA puts them back)
+    int32_t queue_first, queue_count;// items [queue_first, queue_first + queue_count) are handed out at run time
     int32_t batch, total_q, num_units, num_items, num_items_cuda, num_items_tensor;
     int32_t num_split_units, num_ctas_cuda, num_ctas_tensor;
     int32_t num_merge_blocks;

@@ -47,6 +47,11 @@ def test_fixed_chunk_lengths_agree_with_oracle(chunk):
     _, _, plan = run_and_check(wl, what=f"chunk {chunk}", kv_chunk_tokens=chunk)
     if chunk < 1 << 20:
         assert plan.info["num_split_units"] > 0
+    # fixed chunks are dealt to the CTAs statically, and some CTA gets span tiles and warp-body
+    # items: the fused kernel runs both bodies there, one after the other
+    if chunk <= 128:
+        items = plan.items()
+        assert set(items[items["path"] == 1]["cta"].tolist()) & set(items[items["path"] == 0]["cta"].tolist())
 
 
 @pytest.mark.parametrize("Hq", [8, 16])
@@ -59,28 +64,45 @@ def test_cuda_core_path_handles_spans_too(Hq):
     assert plan.info["num_items_tensor"] == 0
 
 
-def test_eight_heads_per_kv_head_decode_rows_take_the_tensor_path():
+def test_eight_heads_per_kv_head():
+    """Default routing with 8 heads per kv head: decode rows (8 columns of the warp body's MMAs) stay on
+    the warp body, the 20-token span (160 rows) takes the span body; tensor_min_rows = 8 sends the
+    decode rows to the span body as well."""
     shape = W.Shape(16, 2, 128, 16)
     wl = W.make_single_step("gqa8", shape, [300, 0, 1500, 77], [1, 1, 1, 20], seed=79)
-    _, _, plan = run_and_check(wl, what="gqa8 decode on tensor cores")
-    assert plan.info["num_items_tensor"] == plan.info["num_items"]
-    _, _, plan = run_and_check(wl, what="gqa8 decode on cuda cores", tensor_min_rows=32)
+    _, _, plan = run_and_check(wl, what="gqa8, default routing")
     assert 0 < plan.info["num_items_tensor"] < plan.info["num_items"]
+    items = plan.items()
+    assert (items[items["path"] == 0]["ntok"] == 1).all() and (items[items["path"] == 1]["seq"] == 3).all()
+    _, _, plan = run_and_check(wl, what="gqa8, every row on the span body", tensor_min_rows=8)
+    assert plan.info["num_items_tensor"] == plan.info["num_items"]
 
 
-def test_decode_rows_on_span_ctas_run_as_narrow_tensor_items():
-    """Default policy, 4 heads per kv head: CTAs that hold span units take decode rows as tensor-core
-    items of 4 rows (cut where the CTA is full), the other CTAs run them on the CUDA-core body."""
+def test_decode_rows_beside_spans_on_few_sms():
+    """Default policy with 12 CTAs: span units on the first CTAs, decode rows queued for whichever CTA
+    is free (span CTAs join the queue when their span tiles are done)."""
     shape = W.Shape(8, 2, 128, 16)
     ctx = [1900, 40, 2500, 3, 700, 1200, 0, 333] + [900 + 37 * i for i in range(24)]
     ql = [40, 1, 1, 9, 1, 64, 1, 1] + [1] * 24
     wl = W.make_single_step("hybrid", shape, ctx, ql, seed=83)
     _, _, plan = run_and_check(wl, what="decode rows beside spans", num_sms=12)
     items = plan.items()
-    tens, cuda = items[items["path"] == 1], items[items["path"] == 0]
-    assert ((tens["ntok"] == 1).sum() > 0) and len(cuda) > 0
-    out_a, lse_a, _ = run_and_check(wl, what="all rows on the CUDA-core body", flags=B.PLAN_NO_TENSOR_PATH)
-    out_b, lse_b, _ = run_and_check(wl, what="all rows on the tensor-core body", tensor_min_rows=1)
+    tens, warp = items[items["path"] == 1], items[items["path"] == 0]
+    assert len(tens) > 0 and (warp["cta"] < 0).sum() > 0
+    assert plan.info["num_split_units"] > 0          # short chunks at the end of the queue: merged in the kernel
+    run_and_check(wl, what="all rows on the warp body", flags=B.PLAN_NO_TENSOR_PATH)
+    run_and_check(wl, what="all rows on the span body", tensor_min_rows=1)
+
+
+def test_short_spans_share_the_columns_of_a_warp_body_unit():
+    """Spans below 32 rows run on the warp body, 8 / G tokens to a unit (2 at 4 heads per kv head, 8 at
+    one), each column with its own causal limit; odd span lengths leave a unit partly empty."""
+    for Hq, Hkv, d in [(8, 2, 128), (4, 4, 64), (2, 1, 128), (16, 2, 64)]:
+        shape = W.Shape(Hq, Hkv, d, 16)
+        wl = W.make_single_step("short", shape, [0, 5, 130, 1000, 16, 255], [3, 7, 2, 5, 1, 6], seed=500 + Hq)
+        _, _, plan = run_and_check(wl, what=f"short spans {Hq}/{Hkv}/{d}")
+        items = plan.items()
+        assert (items["path"] == 0).all() and items["ntok"].max() == min(7, 8 // shape.group)
 
 
 def test_results_are_bitwise_reproducible():
@@ -233,3 +255,40 @@ def test_config2_llama_batch_full_size():
     assert_close(out, lse, ref_out, ref_lse, rows=np.nonzero(~is_app)[0], what="config2 decode rows")
     assert_close(out, lse, ref_out, ref_lse, rows=np.nonzero(is_app)[0], what="config2 append rows")
     assert_close(out, lse, ref_out, ref_lse, what="config2")
+
+
+def test_page_ids_whose_offsets_need_64_bits():
+    """Pages high in a pool of 70 000 pages (4.6 GB): element offsets beyond 2^31 and byte offsets beyond
+    2^32 in the append, in the span body's 16-byte copies and in the warp body's tensor-map
+    coordinates.  Only the pages in use are written on the device; the oracle works on a compact copy
+    of those pages under renumbered ids."""
+    shape = W.Shape(32, 8, 128, 16)
+    small = W.make_single_step("high", shape, [300, 200, 77, 1030], [1, 40, 2, 1], seed=88, spare_pages=0)
+    st = small.steps[0]
+    num_pages = 70000
+    high = (np.random.default_rng(5).permutation(num_pages - 66000)[:small.num_pages] + 66000).astype(np.int32)
+    assert int(high.min()) * shape.page_elems > 2**31
+    pool_dev = torch.empty((num_pages,) + small.kv_pool.shape[1:], dtype=torch.bfloat16, device="cuda")
+    pool_dev[torch.from_numpy(high.astype(np.int64)).cuda()] = to_dev(small.kv_pool)
+    big = W.Workload("high", shape, num_pages, small.kv_pool)
+    st_big = W.Step(st.q_indptr, st.kv_len_before, st.page_indptr, high[st.page_indices], st.q, st.k_new, st.v_new)
+    pool_dev, out, lse, plan = gpu_step(big, st_big, pool_dev=pool_dev)
+    assert 0 < plan.info["num_items_tensor"] < plan.info["num_items"]
+    ref_pool, ref_out, ref_lse = oracle_step(small, st)
+    got = to_bits(pool_dev[torch.from_numpy(high.astype(np.int64)).cuda()])
+    assert np.array_equal(got, ref_pool), "pool differs after append"
+    assert_close(out, lse, ref_out, ref_lse, what="high page ids")
+
+
+def test_sequences_that_share_prefix_pages():
+    """Two sequences (a fork after a common prompt) whose page tables name the same physical pages for
+    their first 20 full pages; each appends into pages of its own.  Reads of shared pages are legal."""
+    shape = W.Shape(8, 2, 128, 16)
+    wl = W.make_single_step("fork", shape, [400, 520, 333, 700], [1, 24, 1, 3], seed=97)
+    st = wl.steps[0]
+    shared = 20
+    for b in (1, 3):      # sequences 1 and 3 start with sequence 0's first 20 pages
+        st.page_indices[st.page_indptr[b]:st.page_indptr[b] + shared] = \
+            st.page_indices[st.page_indptr[0]:st.page_indptr[0] + shared]
+    _, _, plan = run_and_check(wl, what="shared prefix pages", flags=B.PLAN_REJECT_ALIASED_WRITES)
+    assert plan.info["num_items_tensor"] > 0

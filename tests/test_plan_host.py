@@ -59,9 +59,29 @@ def test_cover_with_paused_and_empty_context_sequences(sms):
     check_cover(wl, p)
 
 
-def test_balance_on_the_llama_batch():
-    wl = W.make_config(2, scale=1.0) if False else None
-    # lengths only: build tables without materialising values
+def _queue_checks(p, items, n_sms):
+    """Properties of the run-time queue of warp-body chunks under the default policy."""
+    warp = items[items["path"] == 0]
+    own = warp[warp["cta"] >= 0]
+    queue = warp[warp["cta"] < 0]
+    # a CTA starts on at most one chunk of its own; everything else is handed out at run time
+    assert len(set(own["cta"].tolist())) == len(own) and (queue["cta"] == -1).all()
+    # the list holds the own chunks first, then the queue in the order it is handed out
+    n_own = len(own)
+    assert (warp["cta"][:n_own] >= 0).all()
+    # the long pieces come longest first, the short chunks (cut from few units) at the end
+    tiles = -(-(warp["kv1"] - warp["kv0"]) // 128)
+    units = {}
+    for it, t in zip(warp, tiles):
+        units.setdefault((int(it["seq"]), int(it["kv_head"]), int(it["tok0"])), []).append(int(t))
+    split = {k: v for k, v in units.items() if len(v) > 1}
+    whole_or_long = np.array([t for it, t in zip(warp, tiles)
+                              if len(units[(int(it["seq"]), int(it["kv_head"]), int(it["tok0"]))]) <= 3])
+    assert (np.diff(whole_or_long) <= 0).all()
+    return own, queue, tiles, units, split
+
+
+def test_decode_work_goes_to_a_queue_of_long_pieces_and_short_tail_chunks():
     g = np.random.default_rng(0)
     ctx = g.integers(512, 4097, 32)
     ql = np.ones(32, dtype=np.int64); ql[:8] = g.integers(8, 65, 8)
@@ -72,11 +92,13 @@ def test_balance_on_the_llama_batch():
     p = B.plan_host(shape, int(need.sum()), q_indptr, ctx, page_indptr, page_indices, num_sms=148,
                     flags=B.PLAN_NO_TENSOR_PATH)
     items = p.items()
-    load = np.zeros(p.info["num_ctas_cuda"])
-    np.add.at(load, items["cta"], -(-(items["kv1"] - items["kv0"]) // 128) + 1)
-    assert load.max() <= 1.25 * load.mean() + 2
-    # items of one CTA are contiguous in the list
-    assert (np.diff(items["cta"]) >= 0).all()
+    assert (items["path"] == 0).all()
+    own, queue, tiles, units, split = _queue_checks(p, items, 148)
+    assert len(own) == 148 and len(queue) > 0
+    # about a sixth of the tiles is cut into short chunks; the rest stays in long pieces
+    short = sum(sum(v) for v in split.values() if len(v) > 3)
+    assert 0.1 * tiles.sum() <= short <= 0.3 * tiles.sum()
+    assert len(split) < 0.35 * len(units)
 
 
 def test_plan_is_a_function_of_lengths_only():
@@ -159,10 +181,11 @@ def _llama_lengths(seed=0):
     return ctx, ql, int(need.sum()), q_indptr, page_indptr, page_indices
 
 
-def test_mixed_batch_spans_stay_whole_and_loads_balance():
-    """Default policy on the Llama-shaped mixed batch: every (token, key) pair is covered once, span
-    units are cut only when one is larger than a CTA's share, cuts fall on tile boundaries, and the
-    CTAs' tile counts are balanced."""
+def test_mixed_batch_spans_stay_whole_on_few_ctas_and_decode_rows_are_queued():
+    """Default policy on the Llama-shaped mixed batch: every (token, key) pair is covered once; span
+    units are packed whole onto the first CTAs (a unit of two row tiles that would not fit is divided
+    by rows first, so that few span units need partial rows); the CTAs without span work start
+    on one decode chunk each and the rest of the decode work is queued."""
     ctx, ql, num_pages, q_indptr, page_indptr, page_indices = _llama_lengths()
     shape = W.Shape(32, 8, 128, 16)
     p = B.plan_host(shape, num_pages, q_indptr, ctx, page_indptr, page_indices, num_sms=148)
@@ -179,25 +202,22 @@ def test_mixed_batch_spans_stay_whole_and_loads_balance():
     span = items[items["path"] == 1]
     dec = items[items["path"] == 0]
     assert len(span) and len(dec)
-    assert (span["kv0"] % 128 == 0).all() and (dec["kv0"] % 16 == 0).all()
-    # a CTA runs one body only: where span units sit, decode rows ride along as narrow tensor-core items
-    assert not set(span["cta"].tolist()) & set(dec["cta"].tolist())
-    narrow = span[span["ntok"] * 4 < 32]
-    assert len(narrow) and (narrow["ntok"] == 1).all()
-    wide_ctas = set(span[span["ntok"] * 4 >= 32]["cta"].tolist())
-    assert set(narrow["cta"].tolist()) <= wide_ctas
-    # a span unit covers up to 256 (token, head) rows: 64 tokens at 4 heads per kv head
-    assert span["ntok"].max() <= 64 and (span["tok0"] % 64 == 0).all()
-    wide = span[span["ntok"] * 4 >= 32]
-    units = {(int(it["seq"]), int(it["kv_head"]), int(it["tok0"])) for it in wide}
-    pieces = len(wide) / len(units)
-    assert pieces < 1.6, pieces          # most span units are one item (no partial rows, no merge)
-    # modelled load per CTA in KV tiles (a span tile of two row tiles counts double)
-    load = np.zeros(148)
-    np.add.at(load, span["cta"], -(-(span["kv1"] - span["kv0"]) // 128) * np.where(span["ntok"] * 4 > 128, 2.0, 1.0))
-    np.add.at(load, dec["cta"], -(-(dec["kv1"] - dec["kv0"]) // 96))
-    assert load.max() <= 1.35 * load.mean()
-    assert p.info["launches_attn"] == 2 and p.info["num_split_units"] > 0
+    assert (span["kv0"] % 128 == 0).all() and (dec["kv0"] % 128 == 0).all()
+    # span work sits on CTAs 0 .. used-1, the own decode chunks on the others
+    used = int(span["cta"].max()) + 1
+    assert set(span["cta"].tolist()) == set(range(used)) and 0 < used < 148
+    own = dec[dec["cta"] >= 0]
+    assert set(own["cta"].tolist()) == set(range(used, 148))
+    # span units: at most 256 (token, head) rows, i.e. 64 tokens at 4 heads per kv head, and whole
+    assert span["ntok"].max() <= 64
+    keys = [(int(it["seq"]), int(it["kv_head"]), int(it["tok0"])) for it in span]
+    assert len(keys) < 1.3 * len(set(keys))      # only the longest units are cut by keys as well
+    # decode rows: one token per unit, never on the span body
+    assert (dec["ntok"] == 1).all() and (span["ntok"] * 4 >= 32).all()
+    _queue_checks(p, items, 148)
+    # split decode units are merged inside the attention kernel; only span units cut by keys need
+    # the merge kernel
+    assert p.info["launches_attn"] == (2 if len(keys) > len(set(keys)) else 1) and p.info["num_split_units"] > 0
 
 
 @pytest.mark.parametrize("seed", range(6))
@@ -230,6 +250,36 @@ def test_decode_only_batch_has_no_span_items():
     p = B.plan_host(W.Shape(32, 8, 128, 16), int(need.sum()), q_indptr, ctx, page_indptr, page_indices, num_sms=148)
     items = p.items()
     assert (items["path"] == 0).all() and p.info["num_items_tensor"] == 0
-    load = np.zeros(148)
-    np.add.at(load, items["cta"], -(-(items["kv1"] - items["kv0"]) // 96))
-    assert load.max() <= 1.15 * load.mean() + 1
+    own, queue, tiles, units, split = _queue_checks(p, items, 148)
+    assert len(own) == 148 and p.info["launches_attn"] == 1
+
+
+def test_long_span_units_are_cut_by_keys_and_merged_by_the_merge_kernel():
+    """A span over a context far longer than a CTA's share has to be cut by keys as well."""
+    shape = W.Shape(32, 8, 128, 16)
+    ctx, ql = np.array([60000, 900]), np.array([64, 1])
+    need = -(-(ctx + ql) // 16)
+    q_indptr, page_indptr, page_indices, _ = W.build_step_tables(ctx, ql, 16, np.arange(need.sum()))
+    p = B.plan_host(shape, int(need.sum()), q_indptr, ctx, page_indptr, page_indices, num_sms=148)
+    items = p.items()
+    span = items[items["path"] == 1]
+    keys = [(int(it["seq"]), int(it["kv_head"]), int(it["tok0"])) for it in span]
+    assert len(set(keys)) < len(keys)            # some unit has several chunks
+    assert (span["ntok"] * 4 <= 128).all()      # and the row tiles were divided first
+    assert p.info["launches_attn"] == 2
+
+
+def test_host_workspace_must_be_16_byte_aligned():
+    shape = W.Shape(8, 2, 64, 16)
+    lib = B.load()
+    import ctypes
+    cs, co = B._cshape(shape, 2), B._copts(num_sms=148)
+    cb, keep = B._cbatch([0, 1], [20], [0, 2], [1, 0])
+    ws = np.zeros(1 << 14, dtype=np.int64)
+    base = ws.ctypes.data
+    out = ctypes.c_void_p()
+    ok = base + (-base % 16)
+    assert lib.asynclm_plan(ctypes.byref(cs), ctypes.byref(co), ctypes.byref(cb), ok, 1 << 16, None, 0,
+                            None, ctypes.byref(out)) == 0
+    assert lib.asynclm_plan(ctypes.byref(cs), ctypes.byref(co), ctypes.byref(cb), ok + 8, 1 << 16, None, 0,
+                            None, ctypes.byref(out)) == -1
