@@ -15,6 +15,7 @@
  *     asynclm_plan       (host integer work + one async host->device copy of the plan)
  *     asynclm_kv_append  (scatter the new K/V rows into their page slots)
  *     asynclm_attn_mixed (attention of every new row over its sequence's pages)
+ * or, instead of the last two, asynclm_step, which does both in one launch.
  * A plan depends only on the lengths and the page table, so a multi-layer model builds it once per
  * step and reuses it for every layer's pool.
  *
@@ -219,6 +220,24 @@ int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, const void*
  */
 int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv_pool,
                        void* out, float* lse, void* stream);
+
+/*
+ * The whole step in one call: asynclm_kv_append followed by asynclm_attn_mixed, with the same
+ * arguments, results and bit-exact pool contents, but without a separate append launch.  The
+ * interrupt block still goes to the end of the context first (Section 3.2) and is then processed
+ * with the other sequences' decodes (Section 5.3): every work item of the attention kernel copies
+ * the new K/V rows it is about to read into their page slots itself, right before it fetches the
+ * pages that hold them, so no part of the kernel waits for another, and every new row is written
+ * (each new token attends to itself).  Items that read the same new rows write the same bytes.
+ *
+ *   q             device, bf16 [T][num_q_heads][head_dim]
+ *   k_new, v_new  device, bf16 [T][num_kv_heads][head_dim]
+ *   kv_pool       device, bf16, layout above; written (the new rows) and read
+ *   out, lse      as in asynclm_attn_mixed
+ * Errors: INVALID_ARG, CUDA.
+ */
+int asynclm_step(const asynclm_plan_t* plan, const void* q, const void* k_new, const void* v_new,
+                 void* kv_pool, void* out, float* lse, void* stream);
 
 /*
  * Reads the device status word of the plan's workspace (synchronises `stream`).  *host_out is 0

@@ -20,7 +20,7 @@ EXPORTS = [
     "asynclm_version", "asynclm_strerror", "asynclm_plan_workspace_size", "asynclm_plan",
     "asynclm_plan_get_info", "asynclm_plan_get_items", "asynclm_kv_append", "asynclm_attn_mixed",
     "asynclm_last_device_status", "asynclm_last_cuda_error", "asynclm_attn_mixed_static",
-    "asynclm_static_scratch_bytes",
+    "asynclm_static_scratch_bytes", "asynclm_step",
 ]
 
 PLAN_REJECT_ALIASED_WRITES = 1
@@ -99,6 +99,7 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_kv_append.argtypes = [vp, vp, vp, vp, vp]
     lib.asynclm_attn_mixed.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.asynclm_attn_mixed_static.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.asynclm_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.asynclm_static_scratch_bytes.argtypes = []
     lib.asynclm_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     for name in EXPORTS:
@@ -248,6 +249,14 @@ def asynclm_attn_mixed(plan: Plan, q, kv_pool, out, lse=None, stream=None) -> No
     _check(load().asynclm_attn_mixed(plan.handle, q.data_ptr(), kv_pool.data_ptr(), out.data_ptr(),
                                      None if lse is None else lse.data_ptr(), _stream_ptr(stream)),
            "asynclm_attn_mixed")
+
+
+def asynclm_step(plan: Plan, q, k_new, v_new, kv_pool, out, lse=None, stream=None) -> None:
+    """Append and attention in one launch (asynclm_kv_append + asynclm_attn_mixed)."""
+    _check(load().asynclm_step(plan.handle, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                               kv_pool.data_ptr(), out.data_ptr(),
+                               None if lse is None else lse.data_ptr(), _stream_ptr(stream)),
+           "asynclm_step")
 
 
 def asynclm_attn_mixed_static(plan: Plan, q, kv_pool, out, lse=None, stream=None) -> None:

@@ -72,6 +72,20 @@ extern "C" int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, con
     return cuda_status(launch_lse_merge(plan->dev, out, lse, s));
 }
 
+extern "C" int asynclm_step(const asynclm_plan_t* plan, const void* q, const void* k_new, const void* v_new,
+                            void* kv_pool, void* out, float* lse, void* stream) {
+    if (!runnable(plan)) return ASYNCLM_ERR_INVALID_ARG;
+    if (plan->dev.total_q == 0) return ASYNCLM_OK;
+    if (!q || !k_new || !v_new || !kv_pool || !out || !aligned16(q) || !aligned16(k_new) || !aligned16(v_new) ||
+        !aligned16(kv_pool) || !aligned16(out))
+        return ASYNCLM_ERR_INVALID_ARG;
+    if (int rc = check_plan_device(plan->device)) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    int rc = cuda_status(launch_attention(plan->dev, q, kv_pool, out, lse, s, AppendSrc{k_new, v_new, kv_pool}));
+    if (rc != ASYNCLM_OK) return rc;
+    return cuda_status(launch_lse_merge(plan->dev, out, lse, s));
+}
+
 extern "C" int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out) {
     if (!runnable(plan) || !host_out) return ASYNCLM_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;

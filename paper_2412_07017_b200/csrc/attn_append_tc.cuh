@@ -32,7 +32,11 @@
 //                   of the same keys, and a shared ring lets whichever is due use the free slots.
 //   warp 9          one thread issues all MMAs, a group at a time (P V of its tile, then Q K^T of its
 //                   next tile), so that the groups' softmaxes alternate instead of colliding on the
-//                   exponential unit.  The warp owns the tensor-memory allocation.  (Warp 11 idles.)
+//                   exponential unit.  The warp owns the tensor-memory allocation.
+//   warp 11         idle, except when the kernel appends the step's new K/V rows itself
+//                   (asynclm_step): then it runs ahead of the producers and copies, item by item, the
+//                   new rows the item reads into their page slots; the producers wait for an item's
+//                   rows before they fetch its first tile.
 // All hand-offs are mbarriers with bounded waits; a wait that runs out sets the plan's status word
 // and a CTA-wide abort flag, every role falls through to the common exit, and the tensor memory is
 // released there.
@@ -45,7 +49,7 @@ namespace asynclm {
 namespace tc {
 
 constexpr int kThreads = 384;
-constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10;      // warp 11 idles
+constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10, kAppendWarp = 11;
 constexpr int kD = 128;
 constexpr int kTile = 128;                       // keys per K/V ring slot and query rows per row tile
 constexpr int kSub = 64;                         // keys the softmax handles at a time (half an S tile)
@@ -65,7 +69,8 @@ enum Bar { kQFull = 0, kStats, kOFree, kPFull0, kPvDone0 = kPFull0 + 4, kSFull0 
            kNumBars };
 constexpr uint32_t kOffTmemPtr = kOffBar + 8 * kNumBars;
 constexpr uint32_t kOffAbort = kOffTmemPtr + 8;
-constexpr uint32_t kSmemBytes = kOffAbort + 8 + 1024;
+constexpr uint32_t kOffAppended = kOffAbort + 8;      // items of this CTA whose new K/V rows are in the pool
+constexpr uint32_t kSmemBytes = kOffAppended + 8 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
 // tensor memory columns
@@ -237,14 +242,15 @@ __device__ __forceinline__ TItem load_titem(const Work* rec, bool valid) {
 // The whole kernel body, called by all twelve warps with `smem` 1024-byte aligned.
 template <int G>
 __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
-                                        const __nv_bfloat16* __restrict__ pool,
+                                        const __nv_bfloat16* pool,
                                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
-                                        uint8_t* smem) {
+                                        uint8_t* smem, const AppendSrc& app) {
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar0 = sbase + kOffBar;
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_ptr = (volatile uint32_t*)(smem + kOffTmemPtr);
     volatile int* abort_flag = (volatile int*)(smem + kOffAbort);
+    volatile int* appended = (volatile int*)(smem + kOffAppended);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -267,6 +273,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         for (int s = 0; s < kRing; ++s) { mbar_init(bar(kRingFull0 + s), 32); mbar_init(bar(kRingEmpty0 + s), 1); }
         mbar_init(bar(kMmaDrain), 1);
         *abort_flag = 0;
+        *appended = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
@@ -301,6 +308,22 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
             const TItem after = load_titem(p.works + ii + 2, ii + 2 < i1);
             const int ntiles = (cur.kv_end - cur.kv0 + kTile - 1) / kTile;
+            if (app.k_new != nullptr) {
+                // the item's new K/V rows must be in the pool before its tiles are fetched
+                const long long t_wait = clock64();
+                while (*appended <= ii - i0 && ok) {
+                    __nanosleep(64);
+                    if (*abort_flag) ok = false;
+                    else if (clock64() - t_wait > kWaitCycles) {
+                        *abort_flag = 1;
+                        atomicCAS(p.status, 0, 13);
+                        ok = false;
+                    }
+                }
+                ok = __all_sync(0xffffffffu, ok);
+                __threadfence();
+                if (!ok) break;
+            }
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
                 const int t1 = min(t0 + kGroupTiles, ntiles);
@@ -344,6 +367,18 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         if (!ok && last_pos >= 0) {
             // aborted: let the loads already issued land before shared memory goes away
             asm volatile("cp.async.wait_all;" ::: "memory");
+        }
+      } else if (warp == kAppendWarp) {
+        // ------------------------------------------------------------------ append warp (asynclm_step only)
+        if (app.k_new != nullptr) {
+            pdl_wait();
+            for (int ii = i0; ii < i1; ++ii) {
+                const Work rec = ii == i0 ? *head_work : p.works[ii];
+                append_rows_of_item(p, app, rec, lane);
+                __threadfence();      // the rows are visible device-wide before the count moves
+                __syncwarp();
+                if (lane == 0) *appended = ii - i0 + 1;
+            }
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer

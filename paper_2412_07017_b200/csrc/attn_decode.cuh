@@ -283,26 +283,20 @@ __device__ __forceinline__ void merge_loop(const DevPlan& p, __nv_bfloat16* __re
                                            uint32_t req0, uint32_t reqfree0, volatile int* abort_flag) {
     const int lane = threadIdx.x & 31;
     const int Hq = p.num_q_heads;
-    pdl_wait();
-    for (int k = 0;; ++k) {
-        const int j = k % kMergeReqs;
-        if (!mbar_wait(req0 + 8 * j, (uint32_t)(k / kMergeReqs) & 1u, abort_flag, p.status, 5)) break;
-        const TileDesc d = merge_req[j];
-        __syncwarp();
-        if (lane == 0) mbar_arrive(reqfree0 + 8 * j);
-        if (d.flags & kFlagEnd) break;
-        __threadfence();      // the chunks' rows were written before their counts moved: visible now
+    // merges one unit; dry: everything but the stores (see below)
+    auto merge_unit = [&](const TileDesc& d, bool dry) {
         const int ncols = d.ntok * G;
-        // four consecutive values of one column per lane and position, two positions at a time and up
-        // to eight chunks per pass, all requested together: one round trip to L2 per pass
-        for (int e0 = 4 * lane; e0 < ncols * D; e0 += 256) {
-            float4 acc[2];
-            float mx[2], wsum[2];
-            size_t prow0[2], hh[2];
-            int dd[2];
-            bool on[2];
+        // four consecutive values of one column per lane and position; up to four positions and four
+        // chunks per pass, all requested together: a unit of up to four chunks and 512 values costs
+        // one round trip to L2
+        for (int e0 = 4 * lane; e0 < ncols * D; e0 += 512) {
+            float4 acc[4];
+            float mx[4], wsum[4];
+            size_t prow0[4], hh[4];
+            int dd[4];
+            bool on[4];
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < 4; ++u) {
                 const int e = e0 + 128 * u;
                 on[u] = e < ncols * D;
                 const int col = on[u] ? e / D : 0;
@@ -313,13 +307,13 @@ __device__ __forceinline__ void merge_loop(const DevPlan& p, __nv_bfloat16* __re
                 mx[u] = -INFINITY;
                 wsum[u] = 0.f;
             }
-            for (int c0 = 0; c0 < d.n_chunks; c0 += 8) {
-                float l2[2][8];
-                float4 v[2][8];
+            for (int c0 = 0; c0 < d.n_chunks; c0 += 4) {
+                float l2[4][4];
+                float4 v[4][4];
 #pragma unroll
-                for (int u = 0; u < 2; ++u)
+                for (int u = 0; u < 4; ++u)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int i = 0; i < 4; ++i) {
                         l2[u][i] = -INFINITY;
                         v[u][i] = make_float4(0.f, 0.f, 0.f, 0.f);
                         if (on[u] && c0 + i < d.n_chunks) {
@@ -329,16 +323,16 @@ __device__ __forceinline__ void merge_loop(const DevPlan& p, __nv_bfloat16* __re
                         }
                     }
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     float pm = mx[u];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) pm = fmaxf(pm, l2[u][i]);
+                    for (int i = 0; i < 4; ++i) pm = fmaxf(pm, l2[u][i]);
                     const float rescale = pm == -INFINITY ? 1.f : fast_exp2(mx[u] - pm);      // first pass: exp2(-inf) = 0
                     mx[u] = pm;
                     wsum[u] *= rescale;
                     acc[u].x *= rescale; acc[u].y *= rescale; acc[u].z *= rescale; acc[u].w *= rescale;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
+                    for (int i = 0; i < 4; ++i) {
                         const float w = l2[u][i] == -INFINITY ? 0.f : fast_exp2(l2[u][i] - mx[u]);   // -inf: no visible key there
                         wsum[u] += w;
                         if (w != 0.f) {
@@ -349,17 +343,39 @@ __device__ __forceinline__ void merge_loop(const DevPlan& p, __nv_bfloat16* __re
                 }
             }
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
+            for (int u = 0; u < 4; ++u) {
                 if (!on[u]) continue;
                 const int col = (e0 + 128 * u) / D, tok = col / G;
                 const float inv = 1.f / wsum[u];
                 const size_t hq = (size_t)d.kv_head * G + hh[u];
+                if (dry) continue;
                 *reinterpret_cast<uint2*>(out + ((size_t)(d.out_row + tok) * Hq + hq) * D + dd[u]) =
                     make_uint2(pack_bf16x2(acc[u].x * inv, acc[u].y * inv), pack_bf16x2(acc[u].z * inv, acc[u].w * inv));
                 if (lse != nullptr && dd[u] == 0)
                     lse[(size_t)(d.out_row + tok) * Hq + hq] = (mx[u] + log2f(wsum[u])) * kLn2;
             }
         }
+    };
+    // This code runs once or twice per CTA, at the very end of the step, where every microsecond of
+    // cold instruction fetches shows; so it is run once up front, on partial rows that hold nothing
+    // yet and with the stores left out, while the CTA waits for its first pages anyway.
+    if (p.num_split_units > 0) {
+        TileDesc warm{};
+        warm.ntok = 1;
+        warm.n_chunks = 1;
+        warm.partial_base = 0;
+        merge_unit(warm, true);
+    }
+    pdl_wait();
+    for (int k = 0;; ++k) {
+        const int j = k % kMergeReqs;
+        if (!mbar_wait(req0 + 8 * j, (uint32_t)(k / kMergeReqs) & 1u, abort_flag, p.status, 5)) break;
+        const TileDesc d = merge_req[j];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(reqfree0 + 8 * j);
+        if (d.flags & kFlagEnd) break;
+        __threadfence();      // the chunks' rows were written before their counts moved: visible now
+        merge_unit(d, false);
         if (lane == 0) atomicExch(p.unit_arrivals + d.unit, 0);      // ready for the next launch of this plan
         if (lane == 0) trace_add(7, 1);
     }
@@ -372,7 +388,7 @@ template <int D, int GT>
 __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap* kv_map,
                                             const __nv_bfloat16* __restrict__ q,
                                             __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
-                                            int S, uint8_t* smem) {
+                                            int S, uint8_t* smem, const AppendSrc& app) {
     using Geo = Geometry<D>;
     constexpr int G = GT;
     static_assert(G <= kCols && kCols % G == 0, "heads per kv head must divide the column count");
@@ -448,7 +464,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             return r;
         };
         PItem cur{0, 0, 0, 0, 0, 0, -1, 0, 0, 1, -1};
-        if (i0 < i1) {
+        if (i0 < i1 && app.k_new == nullptr) {      // (with the append fused in, every item passes the fetch warp)
             cur = unpack(head + kHeadWorkCuda);
             pages_cur = head[kHeadPagesCuda + lane];
         }
@@ -549,7 +565,7 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         // it has not started.
         const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
         const int i1 = head[3];
-        int own = head[2] < i1 ? head[2] + 1 : i1;
+        int own = head[2] < i1 && app.k_new == nullptr ? head[2] + 1 : head[2];
         pdl_wait();      // the queue's counter belongs to the launch in front until that has completed
         for (int j = 0;; ++j) {
             if (j > 0 && !mbar_wait(next_free, (uint32_t)(j - 1) & 1u, abort_flag, p.status, 7)) break;
@@ -569,6 +585,18 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                 const int kv0 = __shfl_sync(0xffffffffu, w, 0), kv_end = __shfl_sync(0xffffffffu, w, 1);
                 const int page0 = __shfl_sync(0xffffffffu, w, 7);
                 if (lane < (kv_end - kv0 + kPage - 1) / kPage) pg = __ldg(p.page_indices + page0 + lane);
+                if (app.k_new != nullptr) {
+                    // asynclm_step: the new K/V rows this item reads go into their page slots now; the
+                    // producer's copies (asynchronous proxy) come after the hand-off below
+                    Work rec;
+                    rec.kv0 = kv0; rec.kv_end = kv_end; rec.page0 = page0;
+                    rec.q_row0 = __shfl_sync(0xffffffffu, w, 2);
+                    rec.kv_limit0 = __shfl_sync(0xffffffffu, w, 4);
+                    rec.kv_head = __shfl_sync(0xffffffffu, w, 5);
+                    rec.q_seq0 = __shfl_sync(0xffffffffu, w, 11);
+                    append_rows_of_item(p, app, rec, lane);
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                }
             }
             if (lane < 12) next_item->work[lane] = w;
             next_item->pages[lane] = pg;

@@ -87,4 +87,26 @@ __device__ __forceinline__ size_t pool_row_offset(int64_t page, int which, int k
             (size_t)slot) * (size_t)head_dim;
 }
 
+// Interrupt append inside an attention kernel (paper Section 3.2: the block goes to the end of the
+// context): one warp copies, bit for bit, the new K/V rows of one kv head that an item is about to
+// read, positions [max(kv0, ctx), kv_end) of its sequence, from k_new / v_new into their page slots.
+// Every item does this for the rows it reads itself, so no CTA ever waits for another; items that
+// read the same rows write the same bytes.  `w`: the item's Work record.
+__device__ __forceinline__ void append_rows_of_item(const DevPlan& p, const AppendSrc& app, const Work& w, int lane) {
+    const int ctx = w.kv_limit0 - 1 - (w.q_row0 - w.q_seq0);
+    const int lo = max(w.kv0, ctx);
+    const int vpr = p.head_dim / 8;                       // 16-byte vectors per row
+    const int total = (w.kv_end - lo) * 2 * vpr;
+    const uint4* k_new = reinterpret_cast<const uint4*>(app.k_new);
+    const uint4* v_new = reinterpret_cast<const uint4*>(app.v_new);
+    uint4* pool = reinterpret_cast<uint4*>(app.pool);
+    for (int i = lane; i < total; i += 32) {
+        const int pos = lo + i / (2 * vpr), r = i % (2 * vpr);
+        const int which = r / vpr, vec = r % vpr;
+        const int64_t page = __ldg(p.page_indices + w.page0 + (pos - w.kv0) / kPage);
+        const uint4 val = ldg_nc_v4((which ? v_new : k_new) + ((size_t)(w.q_seq0 + pos - ctx) * p.num_kv_heads + w.kv_head) * vpr + vec);
+        pool[pool_row_offset(page, which, w.kv_head, pos % kPage, p.num_kv_heads, p.head_dim) / 8 + vec] = val;
+    }
+}
+
 }  // namespace asynclm

@@ -9,10 +9,11 @@ namespace asynclm {
 cudaError_t launch_kv_append(const DevPlan& p, const void* k_new, const void* v_new, void* kv_pool,
                              cudaStream_t stream);
 
-// All attention kernels of a step: tensor-core span tiles and CUDA-core decode rows (one fused
-// launch when the step has both), writing final rows to `out` and split rows to the plan's partials.
+// All attention kernels of a step: span tiles and warp-body items (one fused launch when the step
+// has both), writing final rows to `out` and split rows to the plan's partials.  With app.k_new set
+// the kernels first put every new K/V row they are about to read into its page slot themselves.
 cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
-                             cudaStream_t stream);
+                             cudaStream_t stream, AppendSrc app = AppendSrc{nullptr, nullptr, nullptr});
 
 cudaError_t launch_lse_merge(const DevPlan& p, void* out, float* lse, cudaStream_t stream);
 

@@ -398,11 +398,10 @@ void deal_dynamic(std::vector<int>& ids_tensor, const std::vector<int>& ids_warp
     std::stable_sort(pieces_out.begin(), pieces_out.end(), [](const Piece& x, const Piece& y) { return x.cta < y.cta; });
 
     // ---- warp-body chunks.  An item boundary costs time and a split unit costs partial rows and a
-    // merge, so most of the work stays in long pieces: units are taken longest first; the first ones, up
-    // to a sixth of all tiles, are cut into short chunks that go to the END of the queue, where they
-    // even out the CTAs' finishing times (few units, many chunks each: few merges); every other unit
-    // stays whole unless it is longer than two fifths of the step, in which case it is cut into equal
-    // pieces.  The queue holds the long pieces longest first, then the short chunks.
+    // merge, so most of the work stays in long pieces: a few units, a sixth of all tiles, are cut into
+    // short chunks that go to the END of the queue, where they even out the CTAs' finishing times;
+    // every other unit stays whole unless it is longer than two fifths of the step, in which case it is
+    // cut into equal pieces.  The queue holds the long pieces longest first, then the short chunks.
     std::vector<int> warp_order(ids_warp);
     std::stable_sort(warp_order.begin(), warp_order.end(),
                      [&](int x, int y) { return units[x].n_keys > units[y].n_keys; });
@@ -411,21 +410,31 @@ void deal_dynamic(std::vector<int>& ids_tensor, const std::vector<int>& ids_warp
     const int64_t bulk_max = std::max<int64_t>(kMinChunkTiles, hi * 2 / 5 / kWarpCost.tile_ns);
     const int64_t tail_target = warp_tiles / 6;
     const int64_t tail_chunk = std::max<int64_t>(kMinChunkTiles, tail_target / ((int64_t)n_ctas * kTailChunksPerCta));
+    // which units are cut short: first those of up to four chunks (their merge is one round trip to
+    // L2), longest first; longer ones only if that does not give a sixth of the tiles
+    std::vector<char> to_tail(units.size(), 0);
     int64_t tail_tiles = 0;
+    for (int pass = 0; pass < 2 && tail_tiles < tail_target; ++pass)
+        for (int id : warp_order) {
+            const int64_t t = tiles_of(units[id].n_keys, kWarpCost.gran);
+            if (tail_tiles >= tail_target) break;
+            if (to_tail[(size_t)id] || t <= tail_chunk + tail_chunk / 2 || (pass == 0 && t > 4 * tail_chunk)) continue;
+            to_tail[(size_t)id] = 1;
+            tail_tiles += t;
+        }
     for (int id : warp_order) {
         const int64_t t = tiles_of(units[id].n_keys, kWarpCost.gran);
-        const bool to_tail = tail_tiles < tail_target && t > tail_chunk + tail_chunk / 2;
-        const int64_t piece_max = to_tail ? tail_chunk : bulk_max;
+        const bool short_chunks = to_tail[(size_t)id] != 0;
+        const int64_t piece_max = short_chunks ? tail_chunk : bulk_max;
         const int64_t pieces = t <= piece_max + piece_max / 2 ? 1 : (t + piece_max - 1) / piece_max;
         int64_t k0 = 0;
         for (int64_t c = 0; c < pieces; ++c) {
             const int64_t take = t / pieces + (c < t % pieces ? 1 : 0);
             const int64_t k1 = std::min<int64_t>(units[id].n_keys, k0 + take * kWarpCost.gran);
-            (to_tail ? tail : chunks).push_back(Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c});
+            (short_chunks ? tail : chunks).push_back(Item{id, (int32_t)k0, (int32_t)k1, (int32_t)c});
             k0 = k1;
         }
         units[id].u.n_chunks = (int32_t)pieces;
-        if (to_tail) tail_tiles += t;
     }
     auto longer = [](const Item& x, const Item& y) { return x.kv1 - x.kv0 > y.kv1 - y.kv0; };
     std::stable_sort(chunks.begin(), chunks.end(), longer);
@@ -668,7 +677,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
         w.unit = it.unit;
         w.n_chunks = u.n_chunks;
         w.partial_base = u.partial_base;
-        w.pad = 0;
+        w.q_seq0 = q_indptr[u.seq];
         h_works[i] = w;
     }
     for (int c = 0; c < std::max(ctas_cuda, ctas_tensor); ++c) {

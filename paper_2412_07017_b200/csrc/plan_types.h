@@ -45,7 +45,8 @@ struct alignas(16) Work {
     int32_t unit;          // the unit this item is a chunk of
     int32_t n_chunks;      // chunks of that unit
     int32_t partial_base;  // partial row of its chunk 0, token 0 (-1 if unsplit)
-    int32_t pad;
+    int32_t q_seq0;        // global token row of the sequence's first new token (its position is
+                           // ctx = kv_limit0 - 1 - (q_row0 - q_seq0))
 };
 
 // Per persistent CTA, one 384-byte header that holds everything the CTA needs to issue its first
@@ -55,6 +56,14 @@ struct alignas(16) Work {
 // 64-95 those of the first warp-body item.
 constexpr int kHeadWords = 96;
 constexpr int kHeadWorkTensor = 8, kHeadWorkCuda = 20, kHeadPagesTensor = 32, kHeadPagesCuda = 64;
+
+// The new K/V rows of the step, for attention kernels that append them themselves (asynclm_step);
+// k_new == nullptr: the rows are in the pool already.
+struct AppendSrc {
+    const void* k_new;     // bf16 [T][Hkv][d]
+    const void* v_new;
+    void* pool;            // the pool, writable
+};
 
 // Pointers into the device workspace, passed to kernels by value.
 struct DevPlan {

@@ -10,6 +10,10 @@ MAX_ABS = 1e-2      # bf16 in, fp32 accumulate, bf16 out: max |gpu - oracle|
 MEAN_ABS = 1e-3     # mean |gpu - oracle| over all output elements of a step
 LSE_ABS = 1e-3
 
+# "calls": asynclm_kv_append + asynclm_attn_mixed; "step": asynclm_step (one launch).  The parity
+# module runs every test both ways.
+API = "calls"
+
 
 def to_dev(bits: np.ndarray) -> torch.Tensor:
     """uint16 bf16 bit patterns -> cuda bfloat16 tensor of the same shape."""
@@ -32,8 +36,11 @@ def gpu_step(wl, st, pool_dev=None, want_lse=True, sm_scale=0.0, **opts):
                      device="cuda") if want_lse else None
     plan = B.asynclm_plan(wl.shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr,
                           st.page_indices, sm_scale=sm_scale, **opts)
-    B.asynclm_kv_append(plan, kn, vn, pool_dev)
-    B.asynclm_attn_mixed(plan, q, pool_dev, out, lse)
+    if API == "step":
+        B.asynclm_step(plan, q, kn, vn, pool_dev, out, lse)
+    else:
+        B.asynclm_kv_append(plan, kn, vn, pool_dev)
+        B.asynclm_attn_mixed(plan, q, pool_dev, out, lse)
     torch.cuda.synchronize()
     assert B.last_device_status(plan) == 0
     return pool_dev, to_bits(out), (lse.cpu().numpy() if want_lse else None), plan

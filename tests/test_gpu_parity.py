@@ -9,9 +9,18 @@ import torch
 
 from paper_2412_07017_b200 import binding as B
 from paper_2412_07017_b200 import workload as W
+import gpu_util
 from gpu_util import (assert_close, gpu_step, oracle_step, to_bits, to_dev)
 
 pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True, params=["calls", "step"])
+def api(request):
+    """Every test runs through the three calls and through asynclm_step."""
+    gpu_util.API = request.param
+    yield request.param
+    gpu_util.API = "calls"
 
 
 def run_and_check(wl, st=None, what="", **opts):
