@@ -100,12 +100,26 @@ __device__ __forceinline__ void append_rows_of_item(const DevPlan& p, const Appe
     const uint4* k_new = reinterpret_cast<const uint4*>(app.k_new);
     const uint4* v_new = reinterpret_cast<const uint4*>(app.v_new);
     uint4* pool = reinterpret_cast<uint4*>(app.pool);
-    for (int i = lane; i < total; i += 32) {
-        const int pos = lo + i / (2 * vpr), r = i % (2 * vpr);
-        const int which = r / vpr, vec = r % vpr;
-        const int64_t page = __ldg(p.page_indices + w.page0 + (pos - w.kv0) / kPage);
-        const uint4 val = ldg_nc_v4((which ? v_new : k_new) + ((size_t)(w.q_seq0 + pos - ctx) * p.num_kv_heads + w.kv_head) * vpr + vec);
-        pool[pool_row_offset(page, which, w.kv_head, pos % kPage, p.num_kv_heads, p.head_dim) / 8 + vec] = val;
+    // sixteen vectors per lane are requested together, then stored: the copy is a chain of round trips
+    // to memory otherwise
+    constexpr int kBatch = 16;
+    for (int base = lane; base < total; base += 32 * kBatch) {
+        uint4 val[kBatch];
+        size_t dst[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const int i = base + 32 * j;
+            if (i < total) {
+                const int pos = lo + i / (2 * vpr), r = i % (2 * vpr);
+                const int which = r / vpr, vec = r % vpr;
+                const int64_t page = __ldg(p.page_indices + w.page0 + (pos - w.kv0) / kPage);
+                val[j] = ldg_nc_v4((which ? v_new : k_new) + ((size_t)(w.q_seq0 + pos - ctx) * p.num_kv_heads + w.kv_head) * vpr + vec);
+                dst[j] = pool_row_offset(page, which, w.kv_head, pos % kPage, p.num_kv_heads, p.head_dim) / 8 + vec;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j)
+            if (base + 32 * j < total) pool[dst[j]] = val[j];
     }
 }
 
