@@ -249,6 +249,7 @@ def run_gpu(args):
     for _ in range(max(args.warmup, 3)):
         flush.fill_(1)
         step()
+        B.asynclm_step(plan, q, kn, vn, pool, out, None, stream)
     torch.cuda.synchronize()
     assert B.last_device_status(plan) == 0
 

@@ -226,24 +226,23 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 
 // One work item as the kernel sees it (kv_end == 0: no item).
 struct TItem {
-    int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row0, page0, q_seq0;
+    int kv0, kv_end, q_row0, ntok, kv_limit0, kv_head, partial_row0, page0;
 };
 
 // `rec`: a Work record (the planner's array, or the copy of a CTA's first item in its header).
 __device__ __forceinline__ TItem load_titem(const Work* rec, bool valid) {
-    TItem r{0, 0, 0, 0, 0, 0, -1, 0, 0};
+    TItem r{0, 0, 0, 0, 0, 0, -1, 0};
     if (valid) {
         const int4* src = reinterpret_cast<const int4*>(rec);
-        const int4 a = __ldg(src), b = __ldg(src + 1), c = __ldg(src + 2);
+        const int4 a = __ldg(src), b = __ldg(src + 1);
         r.kv0 = a.x; r.kv_end = a.y; r.q_row0 = a.z; r.ntok = a.w;
         r.kv_limit0 = b.x; r.kv_head = b.y; r.partial_row0 = b.z; r.page0 = b.w;
-        r.q_seq0 = c.w;
     }
     return r;
 }
 
 // The whole kernel body, called by all twelve warps with `smem` 1024-byte aligned.
-template <int G>
+template <int G, bool APPEND>
 __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* __restrict__ q,
                                         const __nv_bfloat16* pool,
                                         __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
@@ -311,9 +310,13 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         for (int ii = i0; cur.kv_end > 0 && ok; ++ii) {
             const TItem after = load_titem(p.works + ii + 2, ii + 2 < i1);
             const int ntiles = (cur.kv_end - cur.kv0 + kTile - 1) / kTile;
-            // asynclm_step: the first key position of the item that this step appends; tiles up to it
-            // are fetched at once, the others only when the append warp has put the rows in the pool
-            const int first_new = app.k_new != nullptr ? cur.kv_limit0 - 1 - (cur.q_row0 - cur.q_seq0) : INT_MAX;
+            // APPEND: the first key position of the item that this step appends; tiles up to it are
+            // fetched at once, the others only when the append warp has put the rows in the pool
+            int first_new = INT_MAX;
+            if constexpr (APPEND) {
+                const int q_seq0 = ii == i0 ? head_work->q_seq0 : __ldg(&p.works[ii].q_seq0);
+                first_new = cur.kv_limit0 - 1 - (cur.q_row0 - q_seq0);
+            }
             bool appended_seen = false;
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
@@ -321,21 +324,23 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 for (int t = t0; t < t1 && ok; ++t, ++n) {
                     const int rows = min(kTile, cur.kv_end - (cur.kv0 + t * kTile));
                     const int npages = (rows + kPage - 1) / kPage;
-                    if (!appended_seen && cur.kv0 + t * kTile + rows > first_new) {
-                        const long long t_wait = clock64();
-                        while (*appended <= ii - i0 && ok) {
-                            __nanosleep(64);
-                            if (*abort_flag) ok = false;
-                            else if (clock64() - t_wait > kWaitCycles) {
-                                *abort_flag = 1;
-                                atomicCAS(p.status, 0, 13);
-                                ok = false;
+                    if constexpr (APPEND) {
+                        if (!appended_seen && cur.kv0 + t * kTile + rows > first_new) {
+                            const long long t_wait = clock64();
+                            while (*appended <= ii - i0 && ok) {
+                                __nanosleep(64);
+                                if (*abort_flag) ok = false;
+                                else if (clock64() - t_wait > kWaitCycles) {
+                                    *abort_flag = 1;
+                                    atomicCAS(p.status, 0, 13);
+                                    ok = false;
+                                }
                             }
+                            ok = __all_sync(0xffffffffu, ok);
+                            if (!ok) break;
+                            __threadfence();
+                            appended_seen = true;
                         }
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
-                        __threadfence();
-                        appended_seen = true;
                     }
                     const int pos = which ? ring_pos_v(n) : ring_pos_k(n);
                     const int s = pos % kRing;
@@ -377,7 +382,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         }
       } else if (warp == kAppendWarp) {
         // ------------------------------------------------------------------ append warp (asynclm_step only)
-        if (app.k_new != nullptr) {
+        if constexpr (APPEND) {
             pdl_wait();
             for (int ii = i0; ii < i1; ++ii) {
                 const Work rec = ii == i0 ? *head_work : p.works[ii];

@@ -33,8 +33,6 @@
 #pragma once
 #include <cuda.h>
 
-#include <climits>
-
 #include "common.cuh"
 #include "kernels.h"
 
@@ -386,7 +384,7 @@ __device__ __forceinline__ void merge_loop(const DevPlan& p, __nv_bfloat16* __re
 
 // The whole kernel body: warps 0-7 consume, warp 8 produces, warps 9 and 10 are the epilogue and the
 // merge warp, any further warps of the CTA return at once (the fused kernel has twelve).
-template <int D, int GT>
+template <int D, int GT, bool APPEND>
 __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap* kv_map,
                                             const __nv_bfloat16* __restrict__ q,
                                             __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
@@ -402,7 +400,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
     NextItem* next_item = (NextItem*)(merge_req + kMergeReqs);
     uint64_t* bars = (uint64_t*)(next_item + 1);   // full[S], empty[S], done[kHandoffs], req, reqfree, next full, free
     volatile int* abort_flag = (volatile int*)(bars + 2 * S + kHandoffs + 2 * kMergeReqs + 2);
-    volatile int* appended = abort_flag + 1;     // asynclm_step: items of this CTA whose new K/V rows are in the pool
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -419,7 +416,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         for (int h = 0; h < kHandoffs; ++h) mbar_init(done0 + 8 * h, kWarps);
         for (int j = 0; j < 2 * kMergeReqs + 2; ++j) mbar_init(req0 + 8 * j, 1);
         *abort_flag = 0;
-        *appended = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -454,14 +450,12 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         bool ok = true;
         int taken = 0;
         int pages_cur = 0;
-        int q_seq0_cur = 0;      // global token row of the first new token of the current item's sequence
         // next item from the fetch warp (kv_end == 0: none); also sets pages_cur to its first 32 page ids
         auto take = [&]() {
             PItem r{0, 0, 0, 0, 0, 0, -1, 0, 0, 1, -1};
             ok = mbar_wait(next_full, (uint32_t)taken & 1u, abort_flag, p.status, 6);
             if (ok) {
                 r = unpack(next_item->work);
-                q_seq0_cur = next_item->work[11];
                 pages_cur = next_item->pages[lane];
                 __syncwarp();
                 if (lane == 0) mbar_arrive(next_free);
@@ -470,22 +464,16 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
             return r;
         };
         PItem cur{0, 0, 0, 0, 0, 0, -1, 0, 0, 1, -1};
-        if (i0 < i1) {
+        if (i0 < i1 && !APPEND) {      // (with the append fused in, every item passes the fetch warp)
             cur = unpack(head + kHeadWorkCuda);
-            q_seq0_cur = head[kHeadWorkCuda + 11];
             pages_cur = head[kHeadPagesCuda + lane];
         }
         // The plan was uploaded before the kernel in front of this one started, so all of the above
         // overlaps that kernel's tail; the pool, Q and the queue are touched only from here on.
         pdl_wait();
         if (cur.kv_end == 0) cur = take();      // a CTA that came from span tiles starts on the queue
-        int item_seq = 0;      // items of this CTA so far, in the order the fetch warp appends their rows
         while (cur.kv_end > 0 && ok) {
             const int ntiles = (cur.kv_end - cur.kv0 + kTileTok - 1) / kTileTok;
-            // asynclm_step: the first key position of the item that this step appends; stages up to it
-            // are fetched at once, the others only when the fetch warp has put the rows in the pool
-            const int first_new = app.k_new != nullptr ? cur.kv_limit0 - 1 - (cur.q_row0 - q_seq0_cur) : INT_MAX;
-            bool appended_seen = false;
             for (int t0 = 0; t0 < ntiles && ok; t0 += kGroupTiles) {
                 int pages_nxt = 0;
                 const int t1 = min(t0 + kGroupTiles, ntiles);
@@ -498,22 +486,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                     const int rows = min(kTileTok, cur.kv_end - base);
                     const int npages = (rows + kPage - 1) / kPage;
                     const bool first = t == 0;
-                    if (!appended_seen && base + rows > first_new) {
-                        const long long t_wait = clock64();
-                        while (*appended <= item_seq && ok) {
-                            __nanosleep(64);
-                            if (*abort_flag) ok = false;
-                            else if (clock64() - t_wait > kWaitCycles) {
-                                *abort_flag = 1;
-                                atomicCAS(p.status, 0, 8);
-                                ok = false;
-                            }
-                        }
-                        ok = __all_sync(0xffffffffu, ok);
-                        if (!ok) break;
-                        __threadfence();
-                        appended_seen = true;
-                    }
                     if (lane == 0) {
                         TileDesc d;
                         d.flags = (first ? kFlagFirst : 0) | (t == ntiles - 1 ? kFlagLast : 0);
@@ -551,7 +523,6 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                 }
                 pages_cur = pages_nxt;
             }
-            ++item_seq;
             if (ok) cur = take();
         }
         if (ok) {
@@ -594,19 +565,8 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
         // it has not started.
         const int32_t* head = p.cta_heads + (size_t)blockIdx.x * kHeadWords;
         const int i1 = head[3];
-        int own = head[2] < i1 ? head[2] + 1 : i1;
-        int n_appended = 0;
-        auto append_item = [&](const Work& rec) {
-            // asynclm_step: the new K/V rows the item reads go into their page slots; the producer's
-            // copies (asynchronous proxy) of the stages that hold them wait for the count
-            append_rows_of_item(p, app, rec, lane);
-            asm volatile("fence.proxy.async.global;" ::: "memory");
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) *appended = ++n_appended;
-        };
+        int own = head[2] < i1 && !APPEND ? head[2] + 1 : head[2];
         pdl_wait();      // the queue's counter belongs to the launch in front until that has completed
-        if (app.k_new != nullptr && head[2] < i1) append_item(*reinterpret_cast<const Work*>(head + kHeadWorkCuda));
         for (int j = 0;; ++j) {
             if (j > 0 && !mbar_wait(next_free, (uint32_t)(j - 1) & 1u, abort_flag, p.status, 7)) break;
             int idx = -1;
@@ -625,20 +585,24 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                 const int kv0 = __shfl_sync(0xffffffffu, w, 0), kv_end = __shfl_sync(0xffffffffu, w, 1);
                 const int page0 = __shfl_sync(0xffffffffu, w, 7);
                 if (lane < (kv_end - kv0 + kPage - 1) / kPage) pg = __ldg(p.page_indices + page0 + lane);
+                if constexpr (APPEND) {
+                    // asynclm_step: the new K/V rows this item reads go into their page slots now; the
+                    // producer's copies (asynchronous proxy) come after the hand-off below
+                    Work rec;
+                    rec.kv0 = kv0; rec.kv_end = kv_end; rec.page0 = page0;
+                    rec.q_row0 = __shfl_sync(0xffffffffu, w, 2);
+                    rec.kv_limit0 = __shfl_sync(0xffffffffu, w, 4);
+                    rec.kv_head = __shfl_sync(0xffffffffu, w, 5);
+                    rec.q_seq0 = __shfl_sync(0xffffffffu, w, 11);
+                    append_rows_of_item(p, app, rec, lane);
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                }
             }
             if (lane < 12) next_item->work[lane] = w;
             next_item->pages[lane] = pg;
             __syncwarp();
             if (lane == 0) mbar_arrive(next_full);
             if (idx < 0) break;
-            if (app.k_new != nullptr) {
-                Work rec;
-                rec.kv0 = __shfl_sync(0xffffffffu, w, 0); rec.kv_end = __shfl_sync(0xffffffffu, w, 1);
-                rec.q_row0 = __shfl_sync(0xffffffffu, w, 2); rec.kv_limit0 = __shfl_sync(0xffffffffu, w, 4);
-                rec.kv_head = __shfl_sync(0xffffffffu, w, 5); rec.page0 = __shfl_sync(0xffffffffu, w, 7);
-                rec.q_seq0 = __shfl_sync(0xffffffffu, w, 11);
-                append_item(rec);
-            }
         }
         return;
     }

@@ -26,26 +26,26 @@ __device__ __forceinline__ uint8_t* aligned_smem(uint8_t* raw) {
     return (uint8_t*)(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
 }
 
-template <int D, int G>
+template <int D, int G, bool APPEND>
 __global__ void __launch_bounds__(dec::kThreads, 1)
 attn_decode_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const __nv_bfloat16* __restrict__ q,
                    __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int S, AppendSrc app) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();      // the split-KV merge behind this kernel may start its prologue
     if (threadIdx.x == 0) { trace_mark(0); trace_set(1, 0); trace_set(5, 0); trace_set(6, 0); trace_set(7, 0); }
-    dec::decode_body<D, G>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw), app);
+    dec::decode_body<D, G, APPEND>(p, &kv_map, q, out, lse, S, aligned_smem(smem_raw), app);
 }
 
-template <int G>
+template <int G, bool APPEND>
 __global__ void __launch_bounds__(tc::kThreads, 1)
 attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* pool,
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse, AppendSrc app) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();      // the kernel behind this one may start its prologue; it waits for this grid to complete
-    tc::tc_body<G>(p, q, pool, out, lse, aligned_smem(smem_raw), app);
+    tc::tc_body<G, APPEND>(p, q, pool, out, lse, aligned_smem(smem_raw), app);
 }
 
-template <int G>
+template <int G, bool APPEND>
 __global__ void __launch_bounds__(tc::kThreads, 1)
 attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const __nv_bfloat16* __restrict__ q,
                   const __nv_bfloat16* pool, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
@@ -61,14 +61,14 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
     if (threadIdx.x == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&kv_map));
     if (head[0] == head[1]) {
         // no span tiles for this CTA: straight to its decode rows, without the tensor-memory set-up
-        dec::decode_body<tc::kD, G>(p, &kv_map, q, out, lse, S, smem, app);
+        dec::decode_body<tc::kD, G, APPEND>(p, &kv_map, q, out, lse, S, smem, app);
         return;
     }
-    tc::tc_body<G>(p, q, pool, out, lse, smem, app);
+    tc::tc_body<G, APPEND>(p, q, pool, out, lse, smem, app);
     if (threadIdx.x == 0) trace_mark(1);
     if (head[2] == head[3] && p.queue_count == 0) return;      // nothing left for the warp body
     __syncthreads();      // tensor memory released, shared memory free for the second phase
-    dec::decode_body<tc::kD, G>(p, &kv_map, q, out, lse, S, smem, app);
+    dec::decode_body<tc::kD, G, APPEND>(p, &kv_map, q, out, lse, S, smem, app);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -109,52 +109,52 @@ int decode_stages() {
     return S;
 }
 
-template <int D, int G>
+template <int D, int G, bool APPEND>
 cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                           cudaStream_t stream, AppendSrc app) {
     const int S = decode_stages<D>();
     const size_t smem = dec::smem_bytes<D>(S);
-    cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
     e = make_kv_map(p, pool, &map);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_decode_kernel<D, G>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p, map,
+    return launch_pdl(attn_decode_kernel<D, G, APPEND>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p, map,
                       (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, S, app);
 }
 
-template <int G>
+template <int G, bool APPEND>
 cudaError_t launch_tensor(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                           cudaStream_t stream, AppendSrc app) {
-    cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)tc::kSmemBytes);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_append_tc_kernel<G>, dim3(p.num_ctas_tensor), dim3(tc::kThreads), tc::kSmemBytes, stream,
+    return launch_pdl(attn_append_tc_kernel<G, APPEND>, dim3(p.num_ctas_tensor), dim3(tc::kThreads), tc::kSmemBytes, stream,
                       p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, app);
 }
 
-template <int G>
+template <int G, bool APPEND>
 cudaError_t launch_fused(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                          cudaStream_t stream, AppendSrc app) {
     const int S = decode_stages<tc::kD>();
     const size_t smem = dec::smem_bytes<tc::kD>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD>(S) : tc::kSmemBytes;
-    cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<G, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
     e = make_kv_map(p, pool, &map);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_fused_kernel<G>, dim3(p.num_ctas_cuda), dim3(tc::kThreads), smem, stream, p, map,
+    return launch_pdl(attn_fused_kernel<G, APPEND>, dim3(p.num_ctas_cuda), dim3(tc::kThreads), smem, stream, p, map,
                       (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S, app);
 }
 
-template <int D>
+template <int D, bool APPEND>
 cudaError_t launch_decode_d(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                             cudaStream_t stream, AppendSrc app) {
     switch (p.group) {
-        case 1: return launch_decode<D, 1>(p, q, pool, out, lse, stream, app);
-        case 2: return launch_decode<D, 2>(p, q, pool, out, lse, stream, app);
-        case 4: return launch_decode<D, 4>(p, q, pool, out, lse, stream, app);
-        case 8: return launch_decode<D, 8>(p, q, pool, out, lse, stream, app);
+        case 1: return launch_decode<D, 1, APPEND>(p, q, pool, out, lse, stream, app);
+        case 2: return launch_decode<D, 2, APPEND>(p, q, pool, out, lse, stream, app);
+        case 4: return launch_decode<D, 4, APPEND>(p, q, pool, out, lse, stream, app);
+        case 8: return launch_decode<D, 8, APPEND>(p, q, pool, out, lse, stream, app);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -163,26 +163,29 @@ cudaError_t launch_decode_d(const DevPlan& p, const void* q, const void* pool, v
 
 bool tensor_path_compiled(int head_dim) { return head_dim == tc::kD; }
 
-cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
-                             cudaStream_t stream, AppendSrc app) {
+namespace {
+
+template <bool APPEND>
+cudaError_t launch_attention_impl(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
+                                  cudaStream_t stream, AppendSrc app) {
     const bool has_tensor = p.num_items_tensor > 0, has_cuda = p.num_items_cuda > 0;
     if (has_tensor && p.head_dim != tc::kD) return cudaErrorInvalidValue;
     if (has_tensor && has_cuda && p.num_ctas_tensor == p.num_ctas_cuda) {
         switch (p.group) {
-            case 1: return launch_fused<1>(p, q, kv_pool, out, lse, stream, app);
-            case 2: return launch_fused<2>(p, q, kv_pool, out, lse, stream, app);
-            case 4: return launch_fused<4>(p, q, kv_pool, out, lse, stream, app);
-            case 8: return launch_fused<8>(p, q, kv_pool, out, lse, stream, app);
+            case 1: return launch_fused<1, APPEND>(p, q, kv_pool, out, lse, stream, app);
+            case 2: return launch_fused<2, APPEND>(p, q, kv_pool, out, lse, stream, app);
+            case 4: return launch_fused<4, APPEND>(p, q, kv_pool, out, lse, stream, app);
+            case 8: return launch_fused<8, APPEND>(p, q, kv_pool, out, lse, stream, app);
             default: return cudaErrorInvalidValue;
         }
     }
     if (has_tensor) {
         cudaError_t e;
         switch (p.group) {
-            case 1: e = launch_tensor<1>(p, q, kv_pool, out, lse, stream, app); break;
-            case 2: e = launch_tensor<2>(p, q, kv_pool, out, lse, stream, app); break;
-            case 4: e = launch_tensor<4>(p, q, kv_pool, out, lse, stream, app); break;
-            case 8: e = launch_tensor<8>(p, q, kv_pool, out, lse, stream, app); break;
+            case 1: e = launch_tensor<1, APPEND>(p, q, kv_pool, out, lse, stream, app); break;
+            case 2: e = launch_tensor<2, APPEND>(p, q, kv_pool, out, lse, stream, app); break;
+            case 4: e = launch_tensor<4, APPEND>(p, q, kv_pool, out, lse, stream, app); break;
+            case 8: e = launch_tensor<8, APPEND>(p, q, kv_pool, out, lse, stream, app); break;
             default: e = cudaErrorInvalidValue;
         }
         if (e != cudaSuccess) return e;
@@ -190,11 +193,19 @@ cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_poo
     if (has_cuda) {
         // a decode kernel behind a tensor kernel would have to wait for it to finish (pdl_wait), which
         // is what stream order gives anyway
-        if (p.head_dim == 128) return launch_decode_d<128>(p, q, kv_pool, out, lse, stream, app);
-        if (p.head_dim == 64) return launch_decode_d<64>(p, q, kv_pool, out, lse, stream, app);
+        if (p.head_dim == 128) return launch_decode_d<128, APPEND>(p, q, kv_pool, out, lse, stream, app);
+        if (p.head_dim == 64) return launch_decode_d<64, APPEND>(p, q, kv_pool, out, lse, stream, app);
         return cudaErrorInvalidValue;
     }
     return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_pool, void* out, float* lse,
+                             cudaStream_t stream, AppendSrc app) {
+    return app.k_new != nullptr ? launch_attention_impl<true>(p, q, kv_pool, out, lse, stream, app)
+                                : launch_attention_impl<false>(p, q, kv_pool, out, lse, stream, app);
 }
 
 }  // namespace asynclm
