@@ -247,6 +247,21 @@ int asynclm_step(const asynclm_plan_t* plan, const void* q, const void* k_new, c
 int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out);
 
 /*
+ * Measurement aid (no counterpart in the paper, none of the method's arithmetic): reads n_blocks
+ * pairs of K/V blocks of the pool with plain 16-byte loads, as fast as the GPU can, so that the
+ * attention kernels' rate can be held against a read-only ceiling for the same scattered blocks.
+ *
+ *   kv_pool          device, 16-byte aligned
+ *   k_block_offsets  device, int64 [n_blocks]: byte offset of a K block (one page, one kv head)
+ *   v_delta_bytes    distance from a K block to its V block (num_kv_heads * page_size * head_dim * 2)
+ *   block_bytes      page_size * head_dim * 2
+ *   sink             device, 4 bytes, left alone unless an XOR of all the data hits one chosen value
+ * Errors: INVALID_ARG, CUDA.
+ */
+int asynclm_read_ceiling(const void* kv_pool, const int64_t* k_block_offsets, int64_t n_blocks,
+                         int64_t v_delta_bytes, int32_t block_bytes, void* sink, void* stream);
+
+/*
  * asynclm_attn_mixed with no caller-provided scratch (the paper has no counterpart to this call; it
  * exists for deployment reasons only).
  *

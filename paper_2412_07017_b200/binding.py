@@ -20,7 +20,7 @@ EXPORTS = [
     "asynclm_version", "asynclm_strerror", "asynclm_plan_workspace_size", "asynclm_plan",
     "asynclm_plan_get_info", "asynclm_plan_get_items", "asynclm_kv_append", "asynclm_attn_mixed",
     "asynclm_last_device_status", "asynclm_last_cuda_error", "asynclm_attn_mixed_static",
-    "asynclm_static_scratch_bytes", "asynclm_step",
+    "asynclm_static_scratch_bytes", "asynclm_step", "asynclm_read_ceiling",
 ]
 
 PLAN_REJECT_ALIASED_WRITES = 1
@@ -100,6 +100,7 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_attn_mixed.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.asynclm_attn_mixed_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.asynclm_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.asynclm_read_ceiling.argtypes = [vp, vp, i64, i64, i32, vp, vp]
     lib.asynclm_static_scratch_bytes.argtypes = []
     lib.asynclm_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     for name in EXPORTS:
@@ -257,6 +258,13 @@ def asynclm_step(plan: Plan, q, k_new, v_new, kv_pool, out, lse=None, stream=Non
                                kv_pool.data_ptr(), out.data_ptr(),
                                None if lse is None else lse.data_ptr(), _stream_ptr(stream)),
            "asynclm_step")
+
+
+def asynclm_read_ceiling(kv_pool, k_block_offsets, v_delta_bytes: int, block_bytes: int, sink, stream=None) -> None:
+    """Read-only ceiling probe: plain loads of the listed K/V block pairs (see include/asynclm.h)."""
+    _check(load().asynclm_read_ceiling(kv_pool.data_ptr(), k_block_offsets.data_ptr(),
+                                       int(k_block_offsets.numel()), int(v_delta_bytes), int(block_bytes),
+                                       sink.data_ptr(), _stream_ptr(stream)), "asynclm_read_ceiling")
 
 
 def asynclm_attn_mixed_static(plan: Plan, q, kv_pool, out, lse=None, stream=None) -> None:
