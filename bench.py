@@ -33,7 +33,7 @@ WORKLOAD = "config2-llama3-8b-mixed-batch"       # the configuration the metric 
 WORKLOADS = {2: WORKLOAD, 3: "config3-large-batch-gqa8", 4: "config4-long-context-split-kv"}
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_fused_kernel, one launch on the default
 # workload, from an ncu capture; None whenever the kernel has changed since the counters were taken
-TRAFFIC_BYTES_PER_LAUNCH = None
+TRAFFIC_BYTES_PER_LAUNCH = 325_221_376
 
 
 def measured_peaks():
@@ -272,7 +272,7 @@ def run_gpu(args):
     torch.cuda.synchronize()
     t_wall0 = time.time()
     first = timed_block()
-    blocks = int(min(100, max(1, np.ceil(500.0 / max(float(first.sum()), 1e-3)))))
+    blocks = args.blocks if args.blocks > 0 else int(min(100, max(1, np.ceil(500.0 / max(float(first.sum()), 1e-3)))))
     if world > 1:      # every rank times the same number of blocks
         nb = torch.tensor([blocks], device="cuda")
         dist.all_reduce(nb, op=dist.ReduceOp.MAX)
@@ -542,6 +542,53 @@ def run_replay(args):
     print(json.dumps(line))
 
 
+def run_timeline(args):
+    """Per-CTA timeline of one attention launch of the default workload, from the time-stamp build of
+    the library (build.py --trace: -DASYNCLM_TRACE adds a few globaltimer reads per CTA).  Prints one
+    JSON line; times are microseconds after the first CTA's entry.  Not a benchmark value."""
+    import ctypes
+    from paper_2412_07017_b200 import build as lib_build
+    os.environ["ASYNCLM_LIBRARY"] = lib_build.build(trace=True)
+    import torch
+    from paper_2412_07017_b200 import binding as B
+    from paper_2412_07017_b200 import workload as W
+    torch.cuda.set_device(0)
+    wl = W.make_config(args.config)
+    st, shape = wl.steps[0], wl.shape
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    pool, q, kn, vn = dev(wl.kv_pool), dev(st.q), dev(st.k_new), dev(st.v_new)
+    out = torch.empty((st.total_q, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
+    plan = B.asynclm_plan(shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices)
+    flush = L2Flush(torch)
+    buf = np.zeros((1024, 8), dtype=np.uint64)
+    for k in range(6):
+        flush.fill_(k)
+        B.asynclm_kv_append(plan, kn, vn, pool)
+        B.asynclm_attn_mixed(plan, q, pool, out, None)
+        torch.cuda.synchronize()
+        assert B.load().asynclm_trace_read(ctypes.c_void_p(buf.ctypes.data)) == 0
+    n = plan.info["num_ctas_cuda"]
+    t = buf[:n].astype(np.int64)
+    t0 = t[:, 0].min()
+    us = lambda col: (t[:, col] - t0) / 1e3
+    span = t[:, 1] > 0
+    stats = lambda a: [round(float(x), 1) for x in (a.min(), a.mean(), a.max())] if len(a) else None
+    print(json.dumps({
+        "workload": WORKLOADS.get(args.config, str(args.config)), "ctas": int(n), "span_ctas": int(span.sum()),
+        "entry_us_min_mean_max": stats(us(0)),
+        "span_body_done_us_min_mean_max": stats(us(1)[span]),
+        "first_page_copy_us_mean_ctas_without_span_work": round(float(us(2)[~span].mean()), 1) if (~span).any() else None,
+        "consumers_done_us_min_mean_max": stats(us(4)),
+        "last_warp_done_us_min_mean_max": stats(us(3)),
+        "warp_body_items_per_cta_mean": round(float(t[:, 5].mean()), 1),
+        "warp_body_stages_per_cta_mean": round(float(t[:, 6].mean()), 1),
+        "split_units_merged_per_cta_mean_max": [round(float(t[:, 7].mean()), 2), int(t[:, 7].max())],
+        "plan": {k: plan.info[k] for k in ("num_items", "num_items_tensor", "num_split_units")}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -549,6 +596,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="how many times the block of --steps steps is timed (0 = enough for about 0.5 s of "
+                         "timed GPU work; 1 keeps a profiler capture short)")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4, 5],
                     help="synthetic configuration; 2 is the benchmark, 3 and 4 are for reference, "
                          "5 replays the interrupt trace step by step")
@@ -556,8 +606,13 @@ def main():
                     help="time a decode-only batch instead (exercises attn_decode_kernel alone)")
     ap.add_argument("--spans-only", action="store_true",
                     help="time a batch in which every sequence gets a 64-token span (attn_append_tc_kernel alone)")
+    ap.add_argument("--timeline", action="store_true",
+                    help="print a per-CTA timeline of one attention launch (time-stamp build of the library) "
+                         "instead of benchmarking")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.timeline:
+        run_timeline(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.config == 5:
         run_replay(args)
