@@ -589,6 +589,63 @@ def run_timeline(args):
         "plan": {k: plan.info[k] for k in ("num_items", "num_items_tensor", "num_split_units")}}))
 
 
+def run_trap(args):
+    """Trap handler (paper Section 5.4): measures what the keep / swap / recompute rule needs, for one
+    layer of the Llama-3-8B attention shape: swap-out + swap-in of a sequence of n tokens through pinned
+    host memory (gather kernel, one copy each way) and recomputation of its attention (a span of n
+    tokens over an empty context).  Fits swap (linear) and recompute (quadratic) and prints one JSON line
+    with the fitted model and the decision table.  Not the benchmarked metric."""
+    import torch
+    from paper_2412_07017_b200 import binding as B
+    from paper_2412_07017_b200 import workload as W
+    torch.cuda.set_device(0)
+    shape = W.Shape(32, 8, 128, 16)
+    lens = [256, 512, 1024, 2048, 4096, 8192]
+    num_pages = 2 * max(lens) // 16 + 64
+    page_bytes = shape.page_elems * 2
+    pool = torch.empty((num_pages, 2, shape.num_kv_heads, 16, shape.head_dim), dtype=torch.bfloat16, device="cuda").normal_()
+    perm = np.random.default_rng(1).permutation(num_pages).astype(np.int32)
+    stream = torch.cuda.current_stream()
+    rows = []
+    for n in lens:
+        npg = -(-n // 16)
+        ids_out, ids_in = perm[:npg], perm[npg:2 * npg]
+        staging = torch.empty(B.kv_swap_staging_bytes(shape, num_pages, npg), dtype=torch.uint8, device="cuda")
+        image = torch.empty(npg * page_bytes, dtype=torch.uint8).pin_memory()
+        q = torch.empty((n, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda").normal_()
+        kn = torch.empty((n, shape.num_kv_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda").normal_()
+        out = torch.empty_like(q)
+        plan = B.asynclm_plan(shape, num_pages, [0, n], [0], [0, npg], ids_in)
+        t_swap, t_gather, t_rec = [], [], []
+        for k in range(13):
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            e[0].record(stream)
+            B.asynclm_kv_swap_out(shape, num_pages, ids_out, pool, staging, image, stream)
+            B.asynclm_kv_swap_in(shape, num_pages, ids_in, pool, staging, image, stream)
+            e[1].record(stream)
+            B.asynclm_step(plan, q, kn, kn, pool, out, None, stream)
+            e[2].record(stream)
+            torch.cuda.synchronize()
+            if k >= 3:
+                t_swap.append(e[0].elapsed_time(e[1]) * 1e3)
+                t_rec.append(e[1].elapsed_time(e[2]) * 1e3)
+        rows.append((n, float(np.median(t_swap)), float(np.median(t_rec)), npg * page_bytes))
+    n_arr = np.array([r[0] for r in rows], dtype=np.float64)
+    sw = np.polyfit(n_arr, [r[1] for r in rows], 1)
+    rc = np.polyfit(n_arr, [r[2] for r in rows], 2)
+    model = {"swap_fixed_us": float(sw[1]), "swap_us_per_token": float(sw[0]), "recompute_fixed_us": float(rc[2]),
+             "recompute_us_per_token": float(rc[1]), "recompute_us_per_token2": float(rc[0])}
+    names = {0: "keep", 1: "swap", 2: "recompute"}
+    table = {str(n): {str(w): names[B.asynclm_trap_decide(model, n, w)[0]] for w in (50, 200, 1000, 5000, 100000)}
+             for n in (128, 300, 1024, 4096, 16384)}
+    print(json.dumps({
+        "what": "trap handler: swap-out + swap-in through pinned host memory and attention recompute, one layer, "
+                "32/8 heads, head_dim 128 (us per sequence of n tokens)",
+        "rows_n_swap_us_recompute_us": [[r[0], round(r[1], 1), round(r[2], 1)] for r in rows],
+        "swap_round_trip_gbs": [round(2 * r[3] / (r[1] * 1e-6) / 1e9, 1) for r in rows],
+        "model": model, "decision_by_tokens_then_wait_us": table}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -609,9 +666,13 @@ def main():
     ap.add_argument("--timeline", action="store_true",
                     help="print a per-CTA timeline of one attention launch (time-stamp build of the library) "
                          "instead of benchmarking")
+    ap.add_argument("--trap", action="store_true",
+                    help="measure KV swap and attention recompute times and print the trap handler's cost model")
     args = ap.parse_args()
     if args.timeline:
         run_timeline(args)
+    elif args.trap:
+        run_trap(args)
     elif args.impl == "reference":
         run_reference(args)
     elif args.config == 5:

@@ -228,7 +228,9 @@ int asynclm_attn_mixed(const asynclm_plan_t* plan, const void* q, const void* kv
  * with the other sequences' decodes (Section 5.3): every work item of the attention kernel copies
  * the new K/V rows it is about to read into their page slots itself, right before it fetches the
  * pages that hold them, so no part of the kernel waits for another, and every new row is written
- * (each new token attends to itself).  Items that read the same new rows write the same bytes.
+ * (each new token attends to itself).  Items that read the same new rows write the same bytes; for
+ * a step with a span of more than 64 tokens (the trap handler's recompute, say) that duplication
+ * would dominate, and the call runs the append as a kernel of its own instead.
  *
  *   q             device, bf16 [T][num_q_heads][head_dim]
  *   k_new, v_new  device, bf16 [T][num_kv_heads][head_dim]
@@ -245,6 +247,50 @@ int asynclm_step(const asynclm_plan_t* plan, const void* q, const void* k_new, c
  * ASYNCLM_OK or ASYNCLM_ERR_DEVICE_STATUS / ASYNCLM_ERR_CUDA.
  */
 int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out);
+
+/*
+ * Trap handler data path (Section 5.4, "Trap Handler": a sequence paused by a trap need not hold its
+ * KV cache in GPU memory while it waits).  The swapped form of a sequence is its pages in logical
+ * order, one contiguous image of n_pages * (2 * num_kv_heads * page_size * head_dim * 2) bytes.
+ *
+ * asynclm_kv_swap_out copies page page_ids[j] of the pool to page j of the image: one gather kernel
+ * into `staging`, then ONE device->host copy of the whole image.  asynclm_kv_swap_in is the reverse,
+ * into whatever pages the sequence is given then (page_ids must be distinct): one host->device copy,
+ * one scatter kernel.  Both are bit copies and asynchronous on `stream`; no other byte of the pool or
+ * of the image is written.  A model with several layers calls them once per layer's pool.
+ *
+ *   shape        head shape and pool capacity (page ids are checked against num_pages)
+ *   page_ids     host, int32 [n_pages]; may be reused as soon as the call returns if it is pageable
+ *                memory, and must stay untouched until the stream reaches the copy if it is pinned
+ *   kv_pool      device, layout above
+ *   staging      device, 256-byte aligned, asynclm_kv_swap_staging_bytes(shape, n_pages) bytes, owned
+ *                by the caller (the library allocates nothing)
+ *   host_image   host (pinned recommended), 16-byte aligned, n_pages * page bytes
+ * Errors: INVALID_ARG, PAGE_TABLE (id outside the pool; duplicate id on swap-in), CUDA.
+ */
+size_t asynclm_kv_swap_staging_bytes(const asynclm_shape* shape, int32_t n_pages);
+int asynclm_kv_swap_out(const asynclm_shape* shape, const int32_t* page_ids, int32_t n_pages,
+                        const void* kv_pool, void* staging, void* host_image, void* stream);
+int asynclm_kv_swap_in(const asynclm_shape* shape, const int32_t* page_ids, int32_t n_pages,
+                       void* kv_pool, void* staging, const void* host_image, void* stream);
+
+/*
+ * Trap handler decision (Section 5.4; worked example in Section 6.4, "Trap handling strategy"): swap
+ * time grows linearly and recompute time quadratically with the context length.  The cache is kept
+ * in GPU memory if both exceed the estimated wait until the next interrupt; otherwise the cheaper of
+ * the two is chosen.  Host arithmetic only.  "Recompute" is an asynclm_plan / asynclm_step over the
+ * whole context with kv_len_before = 0; its cost model is fitted by the caller from measurements
+ * (bench.py --trap prints one for the attention part).
+ */
+typedef struct asynclm_trap_model {
+    double swap_fixed_us, swap_us_per_token;
+    double recompute_fixed_us, recompute_us_per_token, recompute_us_per_token2;
+} asynclm_trap_model;
+#define ASYNCLM_TRAP_KEEP      0
+#define ASYNCLM_TRAP_SWAP      1
+#define ASYNCLM_TRAP_RECOMPUTE 2
+int asynclm_trap_decide(const asynclm_trap_model* model, int32_t context_tokens, double wait_us,
+                        int32_t* decision, double* swap_us, double* recompute_us);
 
 /*
  * Measurement aid (no counterpart in the paper, none of the method's arithmetic): reads n_blocks

@@ -20,8 +20,11 @@ EXPORTS = [
     "asynclm_version", "asynclm_strerror", "asynclm_plan_workspace_size", "asynclm_plan",
     "asynclm_plan_get_info", "asynclm_plan_get_items", "asynclm_kv_append", "asynclm_attn_mixed",
     "asynclm_last_device_status", "asynclm_last_cuda_error", "asynclm_attn_mixed_static",
-    "asynclm_static_scratch_bytes", "asynclm_step", "asynclm_read_ceiling",
+    "asynclm_static_scratch_bytes", "asynclm_step", "asynclm_read_ceiling", "asynclm_kv_swap_staging_bytes",
+    "asynclm_kv_swap_out", "asynclm_kv_swap_in", "asynclm_trap_decide",
 ]
+
+TRAP_KEEP, TRAP_SWAP, TRAP_RECOMPUTE = 0, 1, 2
 
 PLAN_REJECT_ALIASED_WRITES = 1
 PLAN_NO_TENSOR_PATH = 2
@@ -44,6 +47,11 @@ class CShape(ctypes.Structure):
 class CPlanOptions(ctypes.Structure):
     _fields_ = [("num_sms", ctypes.c_int32), ("kv_chunk_tokens", ctypes.c_int32),
                 ("tensor_min_rows", ctypes.c_int32), ("flags", ctypes.c_int32)]
+
+
+class CTrapModel(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in ("swap_fixed_us", "swap_us_per_token", "recompute_fixed_us",
+                                               "recompute_us_per_token", "recompute_us_per_token2")]
 
 
 class CBatch(ctypes.Structure):
@@ -101,12 +109,20 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_attn_mixed_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.asynclm_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.asynclm_read_ceiling.argtypes = [vp, vp, i64, i64, i32, vp, vp]
+    lib.asynclm_kv_swap_staging_bytes.argtypes = [ctypes.POINTER(CShape), i32]
+    lib.asynclm_kv_swap_out.argtypes = [ctypes.POINTER(CShape), vp, i32, vp, vp, vp, vp]
+    lib.asynclm_kv_swap_in.argtypes = [ctypes.POINTER(CShape), vp, i32, vp, vp, vp, vp]
+    lib.asynclm_trap_decide.argtypes = [ctypes.POINTER(CTrapModel), i32, ctypes.c_double,
+                                        ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double),
+                                        ctypes.POINTER(ctypes.c_double)]
     lib.asynclm_static_scratch_bytes.argtypes = []
     lib.asynclm_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     for name in EXPORTS:
-        if name not in ("asynclm_strerror", "asynclm_last_cuda_error", "asynclm_static_scratch_bytes"):
+        if name not in ("asynclm_strerror", "asynclm_last_cuda_error", "asynclm_static_scratch_bytes",
+                        "asynclm_kv_swap_staging_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     lib.asynclm_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.asynclm_kv_swap_staging_bytes.restype = ctypes.c_size_t
     _lib = lib
     return lib
 
@@ -258,6 +274,36 @@ def asynclm_step(plan: Plan, q, k_new, v_new, kv_pool, out, lse=None, stream=Non
                                kv_pool.data_ptr(), out.data_ptr(),
                                None if lse is None else lse.data_ptr(), _stream_ptr(stream)),
            "asynclm_step")
+
+
+def kv_swap_staging_bytes(shape, num_pages: int, n_pages: int) -> int:
+    cs = _cshape(shape, num_pages)
+    return int(load().asynclm_kv_swap_staging_bytes(ctypes.byref(cs), int(n_pages)))
+
+
+def asynclm_kv_swap_out(shape, num_pages: int, page_ids, kv_pool, staging, host_image, stream=None) -> None:
+    """Gather the pages `page_ids` (host ints) of kv_pool into host_image (pinned tensor) via `staging`."""
+    ids, ptr = _i32(page_ids)
+    cs = _cshape(shape, num_pages)
+    _check(load().asynclm_kv_swap_out(ctypes.byref(cs), ptr, len(ids), kv_pool.data_ptr(), staging.data_ptr(),
+                                      host_image.data_ptr(), _stream_ptr(stream)), "asynclm_kv_swap_out")
+
+
+def asynclm_kv_swap_in(shape, num_pages: int, page_ids, kv_pool, staging, host_image, stream=None) -> None:
+    """Scatter host_image (pinned tensor) into the pages `page_ids` (host ints) of kv_pool via `staging`."""
+    ids, ptr = _i32(page_ids)
+    cs = _cshape(shape, num_pages)
+    _check(load().asynclm_kv_swap_in(ctypes.byref(cs), ptr, len(ids), kv_pool.data_ptr(), staging.data_ptr(),
+                                     host_image.data_ptr(), _stream_ptr(stream)), "asynclm_kv_swap_in")
+
+
+def asynclm_trap_decide(model: dict, context_tokens: int, wait_us: float):
+    """(decision, swap_us, recompute_us) of the keep / swap / recompute rule."""
+    cm = CTrapModel(*(float(model[n]) for n, _ in CTrapModel._fields_))
+    dec, s, r = ctypes.c_int32(-1), ctypes.c_double(0), ctypes.c_double(0)
+    _check(load().asynclm_trap_decide(ctypes.byref(cm), int(context_tokens), float(wait_us), ctypes.byref(dec),
+                                      ctypes.byref(s), ctypes.byref(r)), "asynclm_trap_decide")
+    return int(dec.value), float(s.value), float(r.value)
 
 
 def asynclm_read_ceiling(kv_pool, k_block_offsets, v_delta_bytes: int, block_bytes: int, sink, stream=None) -> None:

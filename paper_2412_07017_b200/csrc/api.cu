@@ -43,6 +43,9 @@ extern "C" const char* asynclm_strerror(int status) {
     }
 }
 
+// Longest span for which asynclm_step appends inside the attention kernel.
+constexpr int kStepFusedMaxSpan = 64;
+
 static bool runnable(const asynclm_plan_t* plan) {
     return plan && plan->magic == kPlanMagic && !plan->host_only;
 }
@@ -81,7 +84,17 @@ extern "C" int asynclm_step(const asynclm_plan_t* plan, const void* q, const voi
         return ASYNCLM_ERR_INVALID_ARG;
     if (int rc = check_plan_device(plan->device)) return rc;
     cudaStream_t s = (cudaStream_t)stream;
-    int rc = cuda_status(launch_attention(plan->dev, q, kv_pool, out, lse, s, AppendSrc{k_new, v_new, kv_pool}));
+    int rc;
+    if (plan->max_q_len > kStepFusedMaxSpan) {
+        // In the fused kernel every item copies the new rows it reads, so the units of one long span
+        // copy its first rows again and again (quadratic in the span length): beyond a few hundred
+        // tokens the separate append kernel, which copies every row once, is the better first half.
+        rc = cuda_status(launch_kv_append(plan->dev, k_new, v_new, kv_pool, s));
+        if (rc != ASYNCLM_OK) return rc;
+        rc = cuda_status(launch_attention(plan->dev, q, kv_pool, out, lse, s));
+    } else {
+        rc = cuda_status(launch_attention(plan->dev, q, kv_pool, out, lse, s, AppendSrc{k_new, v_new, kv_pool}));
+    }
     if (rc != ASYNCLM_OK) return rc;
     return cuda_status(launch_lse_merge(plan->dev, out, lse, s));
 }

@@ -717,6 +717,7 @@ extern "C" int asynclm_plan(const asynclm_shape* shape, const asynclm_plan_optio
     plan->h_item_cta = h_item_cta;
     plan->h_kv_len_before = (const int32_t*)(hb + L.off_kv_len);
     plan->h_units_path_split = n_items_cuda;
+    for (int b = 0; b < B; ++b) plan->max_q_len = std::max(plan->max_q_len, q_indptr[b + 1] - q_indptr[b]);
 
     char* db = (char*)dev_ws;
     DevPlan& d = plan->dev;

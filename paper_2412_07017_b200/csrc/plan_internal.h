@@ -34,4 +34,5 @@ struct asynclm_plan_s {
     int32_t h_units_path_split;   // items [0, this) are CUDA-core items, the rest tensor items
     int32_t device;
     int32_t host_only;
+    int32_t max_q_len;            // longest span of the step
 };
