@@ -293,6 +293,26 @@ int asynclm_trap_decide(const asynclm_trap_model* model, int32_t context_tokens,
                         int32_t* decision, double* swap_us, double* recompute_us);
 
 /*
+ * Latency model (Section 6.3, "Latency Analysis", and Appendix A) for n independent function calls
+ * with token-generation latency gen[i] > 0 and execution time exec[i] > 0 (any one unit of time):
+ *     l_sync     = sum gen + sum exec                  calls generated and executed one after the other
+ *     l_sync_par = sum gen + max exec                  generated in sequence, executed concurrently
+ *     l_async    = max_i (gen[o_1] + .. + gen[o_i] + exec[o_i])   for the longest-execution-first order o,
+ * which is the paper's max_f (E(f) + sum of G over pred(f)), and speedup_estimate = 1 + mean exec /
+ * mean gen (Theorem 6.2).  lpt_order (host, [n], may be NULL) receives o.
+ * asynclm_async_latency_of_order evaluates the same completion times for any generation order
+ * (a permutation of 0..n-1); completion[i] (host, [n], may be NULL) is when call i returns, i.e.
+ * when its interrupt becomes available.  Host arithmetic only.  Errors: INVALID_ARG.
+ */
+typedef struct asynclm_latency {
+    double l_sync, l_sync_par, l_async, speedup_estimate;
+} asynclm_latency;
+int asynclm_latency_model(const double* gen, const double* exec, int32_t n, asynclm_latency* out,
+                          int32_t* lpt_order);
+int asynclm_async_latency_of_order(const double* gen, const double* exec, const int32_t* order, int32_t n,
+                                   double* latency, double* completion);
+
+/*
  * Measurement aid (no counterpart in the paper, none of the method's arithmetic): reads n_blocks
  * pairs of K/V blocks of the pool with plain 16-byte loads, as fast as the GPU can, so that the
  * attention kernels' rate can be held against a read-only ceiling for the same scattered blocks.

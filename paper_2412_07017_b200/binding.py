@@ -21,7 +21,8 @@ EXPORTS = [
     "asynclm_plan_get_info", "asynclm_plan_get_items", "asynclm_kv_append", "asynclm_attn_mixed",
     "asynclm_last_device_status", "asynclm_last_cuda_error", "asynclm_attn_mixed_static",
     "asynclm_static_scratch_bytes", "asynclm_step", "asynclm_read_ceiling", "asynclm_kv_swap_staging_bytes",
-    "asynclm_kv_swap_out", "asynclm_kv_swap_in", "asynclm_trap_decide",
+    "asynclm_kv_swap_out", "asynclm_kv_swap_in", "asynclm_trap_decide", "asynclm_latency_model",
+    "asynclm_async_latency_of_order",
 ]
 
 TRAP_KEEP, TRAP_SWAP, TRAP_RECOMPUTE = 0, 1, 2
@@ -52,6 +53,10 @@ class CPlanOptions(ctypes.Structure):
 class CTrapModel(ctypes.Structure):
     _fields_ = [(n, ctypes.c_double) for n in ("swap_fixed_us", "swap_us_per_token", "recompute_fixed_us",
                                                "recompute_us_per_token", "recompute_us_per_token2")]
+
+
+class CLatency(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in ("l_sync", "l_sync_par", "l_async", "speedup_estimate")]
 
 
 class CBatch(ctypes.Structure):
@@ -112,6 +117,8 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_kv_swap_staging_bytes.argtypes = [ctypes.POINTER(CShape), i32]
     lib.asynclm_kv_swap_out.argtypes = [ctypes.POINTER(CShape), vp, i32, vp, vp, vp, vp]
     lib.asynclm_kv_swap_in.argtypes = [ctypes.POINTER(CShape), vp, i32, vp, vp, vp, vp]
+    lib.asynclm_latency_model.argtypes = [vp, vp, i32, ctypes.POINTER(CLatency), vp]
+    lib.asynclm_async_latency_of_order.argtypes = [vp, vp, vp, i32, ctypes.POINTER(ctypes.c_double), vp]
     lib.asynclm_trap_decide.argtypes = [ctypes.POINTER(CTrapModel), i32, ctypes.c_double,
                                         ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double),
                                         ctypes.POINTER(ctypes.c_double)]
@@ -304,6 +311,31 @@ def asynclm_trap_decide(model: dict, context_tokens: int, wait_us: float):
     _check(load().asynclm_trap_decide(ctypes.byref(cm), int(context_tokens), float(wait_us), ctypes.byref(dec),
                                       ctypes.byref(s), ctypes.byref(r)), "asynclm_trap_decide")
     return int(dec.value), float(s.value), float(r.value)
+
+
+def asynclm_latency_model(gen, exe) -> dict:
+    """Closed forms of Section 6.3 for independent calls (gen, exe: positive floats per call)."""
+    g = np.ascontiguousarray(gen, dtype=np.float64)
+    e = np.ascontiguousarray(exe, dtype=np.float64)
+    out = CLatency()
+    order = np.zeros(max(len(g), 1), dtype=np.int32)
+    _check(load().asynclm_latency_model(g.ctypes.data, e.ctypes.data, len(g), ctypes.byref(out), order.ctypes.data),
+           "asynclm_latency_model")
+    return {"l_sync": out.l_sync, "l_sync_par": out.l_sync_par, "l_async": out.l_async,
+            "speedup_estimate": out.speedup_estimate, "lpt_order": order[:len(g)]}
+
+
+def asynclm_async_latency_of_order(gen, exe, order):
+    """(latency, completion time of every call) when the calls are generated in `order`."""
+    g = np.ascontiguousarray(gen, dtype=np.float64)
+    e = np.ascontiguousarray(exe, dtype=np.float64)
+    o = np.ascontiguousarray(order, dtype=np.int32)
+    lat = ctypes.c_double(0)
+    done = np.zeros(max(len(g), 1), dtype=np.float64)
+    _check(load().asynclm_async_latency_of_order(g.ctypes.data, e.ctypes.data, o.ctypes.data, len(g),
+                                                 ctypes.byref(lat), done.ctypes.data),
+           "asynclm_async_latency_of_order")
+    return float(lat.value), done[:len(g)]
 
 
 def asynclm_read_ceiling(kv_pool, k_block_offsets, v_delta_bytes: int, block_bytes: int, sink, stream=None) -> None:
