@@ -646,6 +646,38 @@ def run_trap(args):
         "model": model, "decision_by_tokens_then_wait_us": table}))
 
 
+def run_monitor(args):
+    """Token monitor (paper Section 5.1): masked greedy selection + CML state advance over bf16 logits of
+    the Llama-3 vocabulary (128 256) for 256 sequences; bound by HBM (one read of the logits).  Prints one
+    JSON line.  Not the benchmarked metric."""
+    import torch
+    from paper_2412_07017_b200 import binding as B
+    torch.cuda.set_device(0)
+    batch, vocab = 256, 128256
+    logits = torch.empty((batch, vocab), dtype=torch.bfloat16, device="cuda").normal_()
+    special = {"CALL": 128011, "INTR": 128012, "TRAP": 128013, "END": 128014, "HEAD": 128015}
+    state = torch.from_numpy(np.random.default_rng(0).integers(0, 4, batch).astype(np.int32)).cuda()
+    tok, nxt, fl = (torch.empty_like(state) for _ in range(3))
+    flush = L2Flush(torch)
+    stream = torch.cuda.current_stream()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(50)]
+    for k in range(55):
+        flush.fill_(k & 0xff)
+        if k >= 5:
+            ev[k - 5][0].record(stream)
+        B.asynclm_token_monitor_step(logits, special, state, tok, nxt, fl, stream)
+        if k >= 5:
+            ev[k - 5][1].record(stream)
+    torch.cuda.synchronize()
+    us = float(np.median([e[0].elapsed_time(e[1]) for e in ev])) * 1e3
+    peak, kind = measured_peaks()
+    nbytes = batch * vocab * 2
+    print(json.dumps({"what": "token monitor step, 256 sequences x 128256 bf16 logits", "us_per_step": us,
+                      "roofline": {"bound": "hbm", "achieved": nbytes / us / 1e3, "peak": peak, "peak_kind": kind,
+                                   "unit": "GB/s", "frac": nbytes / us / 1e3 / peak, "algorithmic_bytes": nbytes},
+                      "l2": L2Flush.NOTE}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -668,8 +700,12 @@ def main():
                          "instead of benchmarking")
     ap.add_argument("--trap", action="store_true",
                     help="measure KV swap and attention recompute times and print the trap handler's cost model")
+    ap.add_argument("--monitor", action="store_true",
+                    help="time the token monitor's masked selection kernel instead")
     args = ap.parse_args()
-    if args.timeline:
+    if args.monitor:
+        run_monitor(args)
+    elif args.timeline:
         run_timeline(args)
     elif args.trap:
         run_trap(args)

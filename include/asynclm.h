@@ -293,6 +293,40 @@ int asynclm_trap_decide(const asynclm_trap_model* model, int32_t context_tokens,
                         int32_t* decision, double* swap_us, double* recompute_us);
 
 /*
+ * Token monitor's hook into next-token selection (Section 5.1, "Token Monitor"; CML is Section 3): for
+ * every sequence b, the allowed token with the largest logit is chosen (the lowest id among equal
+ * logits; a NaN logit is never chosen) and the sequence's CML state advances.  Allowed tokens by state:
+ *     0 TEXT  outside a block : ordinary tokens, [CALL], [TRAP]
+ *     1 CALL  after [CALL]    : ordinary tokens (identifier or the call itself), [HEAD], [END]
+ *     2 BODY  after [HEAD]    : ordinary tokens, [END]
+ *     3 TRAP  after [TRAP]    : [END] only          ([TRAP][END] is the whole trap)
+ * [INTR] is allowed nowhere: interrupts are injected by the system (Section 3.2), never generated.
+ * flags_out: ASYNCLM_MONITOR_CALL when this token closed a function-call block (the executor is to be
+ * notified), ASYNCLM_MONITOR_TRAP when it closed a trap (the trap handler is), ASYNCLM_MONITOR_CRITICAL
+ * while the sequence is inside a function-call block after this token (interrupts are deferred).
+ * Greedy selection is this library's reading: the paper leaves the sampling rule to the model's
+ * decoding settings.
+ *
+ *   logits      device, [batch][row_stride] of bf16 (dtype 0) or fp32 (dtype 1), 16-byte aligned rows
+ *   tokens      the five CML token ids (distinct, inside the vocabulary)
+ *   state_in    device, int32 [batch]; token_out / state_out / flags_out device, int32 [batch]
+ *               (state_out may alias state_in)
+ * One kernel on `stream`; vocab * element size bytes are read per sequence.  Errors: INVALID_ARG, CUDA.
+ */
+typedef struct asynclm_cml_tokens {
+    int32_t call, intr, trap, end, head;
+} asynclm_cml_tokens;
+#define ASYNCLM_DTYPE_BF16 0
+#define ASYNCLM_DTYPE_F32  1
+#define ASYNCLM_MONITOR_CALL     1
+#define ASYNCLM_MONITOR_TRAP     2
+#define ASYNCLM_MONITOR_CRITICAL 4
+int asynclm_token_monitor_step(const void* logits, int32_t dtype, int32_t batch, int32_t vocab,
+                               int64_t row_stride, const asynclm_cml_tokens* tokens,
+                               const int32_t* state_in, int32_t* token_out, int32_t* state_out,
+                               int32_t* flags_out, void* stream);
+
+/*
  * Latency model (Section 6.3, "Latency Analysis", and Appendix A) for n independent function calls
  * with token-generation latency gen[i] > 0 and execution time exec[i] > 0 (any one unit of time):
  *     l_sync     = sum gen + sum exec                  calls generated and executed one after the other

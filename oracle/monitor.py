@@ -10,7 +10,7 @@ CML as the model may generate it (Section 3.1-3.2):
     [CALL] {function call} [END]          [CALL] {id} [HEAD] {function call} [END]          [TRAP] [END]
 States: TEXT (outside a block), CALL (after [CALL], no [HEAD] yet), BODY (after [HEAD]), TRAP (after
 [TRAP]).  Decoding here is greedy: the allowed token with the largest logit, the lowest id among equals;
-NaN logits are never chosen.  The paper does not fix a sampling rule; this reading is recorded in
+NaN logits are never chosen; if no allowed token has a logit above -inf, the lowest allowed id is taken.  The paper does not fix a sampling rule; this reading is recorded in
 the design doc.  Nothing here imports, or is imported by, the CUDA package.
 """
 from __future__ import annotations
@@ -67,6 +67,9 @@ def step(logits: np.ndarray, states, special: dict):
     for b in range(B):
         ok = allowed(int(states[b]), special, V) & ~np.isnan(logits[b])
         cand = np.where(ok, logits[b], -np.inf)
-        toks[b] = int(np.argmax(cand))             # first index of the maximum
+        if np.isneginf(cand).all():
+            toks[b] = int(np.argmax(allowed(int(states[b]), special, V)))      # nothing to compare: lowest allowed id
+        else:
+            toks[b] = int(np.argmax(cand))         # first index of the maximum
         nxts[b], flags[b] = advance(int(states[b]), int(toks[b]), special)
     return toks, nxts, flags
