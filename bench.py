@@ -658,6 +658,7 @@ def run_monitor(args):
     special = {"CALL": 128011, "INTR": 128012, "TRAP": 128013, "END": 128014, "HEAD": 128015}
     state = torch.from_numpy(np.random.default_rng(0).integers(0, 4, batch).astype(np.int32)).cuda()
     tok, nxt, fl = (torch.empty_like(state) for _ in range(3))
+    ws = torch.zeros(B.token_monitor_workspace_bytes(batch), dtype=torch.uint8, device="cuda")
     flush = L2Flush(torch)
     stream = torch.cuda.current_stream()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(50)]
@@ -665,7 +666,7 @@ def run_monitor(args):
         flush.fill_(k & 0xff)
         if k >= 5:
             ev[k - 5][0].record(stream)
-        B.asynclm_token_monitor_step(logits, special, state, tok, nxt, fl, stream)
+        B.asynclm_token_monitor_step(logits, special, state, tok, nxt, fl, ws, stream)
         if k >= 5:
             ev[k - 5][1].record(stream)
     torch.cuda.synchronize()

@@ -311,7 +311,11 @@ int asynclm_trap_decide(const asynclm_trap_model* model, int32_t context_tokens,
  *   tokens      the five CML token ids (distinct, inside the vocabulary)
  *   state_in    device, int32 [batch]; token_out / state_out / flags_out device, int32 [batch]
  *               (state_out may alias state_in)
- * One kernel on `stream`; vocab * element size bytes are read per sequence.  Errors: INVALID_ARG, CUDA.
+ *   workspace   device, 16-byte aligned, asynclm_token_monitor_workspace_bytes(batch) bytes, owned by
+ *               the caller and all zero before the first call; every call leaves it all zero again (the
+ *               slices of a row meet there), so calls that share it must not overlap on the GPU
+ * One kernel on `stream`; vocab * element size bytes are read per sequence; batch <= 65535.
+ * Errors: INVALID_ARG, CUDA.
  */
 typedef struct asynclm_cml_tokens {
     int32_t call, intr, trap, end, head;
@@ -321,10 +325,11 @@ typedef struct asynclm_cml_tokens {
 #define ASYNCLM_MONITOR_CALL     1
 #define ASYNCLM_MONITOR_TRAP     2
 #define ASYNCLM_MONITOR_CRITICAL 4
+size_t asynclm_token_monitor_workspace_bytes(int32_t batch);
 int asynclm_token_monitor_step(const void* logits, int32_t dtype, int32_t batch, int32_t vocab,
                                int64_t row_stride, const asynclm_cml_tokens* tokens,
                                const int32_t* state_in, int32_t* token_out, int32_t* state_out,
-                               int32_t* flags_out, void* stream);
+                               int32_t* flags_out, void* workspace, void* stream);
 
 /*
  * Latency model (Section 6.3, "Latency Analysis", and Appendix A) for n independent function calls

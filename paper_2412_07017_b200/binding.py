@@ -22,7 +22,7 @@ EXPORTS = [
     "asynclm_last_device_status", "asynclm_last_cuda_error", "asynclm_attn_mixed_static",
     "asynclm_static_scratch_bytes", "asynclm_step", "asynclm_read_ceiling", "asynclm_kv_swap_staging_bytes",
     "asynclm_kv_swap_out", "asynclm_kv_swap_in", "asynclm_trap_decide", "asynclm_latency_model",
-    "asynclm_async_latency_of_order", "asynclm_token_monitor_step",
+    "asynclm_async_latency_of_order", "asynclm_token_monitor_step", "asynclm_token_monitor_workspace_bytes",
 ]
 
 TRAP_KEEP, TRAP_SWAP, TRAP_RECOMPUTE = 0, 1, 2
@@ -123,7 +123,8 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_kv_swap_in.argtypes = [ctypes.POINTER(CShape), vp, i32, vp, vp, vp, vp]
     lib.asynclm_latency_model.argtypes = [vp, vp, i32, ctypes.POINTER(CLatency), vp]
     lib.asynclm_async_latency_of_order.argtypes = [vp, vp, vp, i32, ctypes.POINTER(ctypes.c_double), vp]
-    lib.asynclm_token_monitor_step.argtypes = [vp, i32, i32, i32, i64, ctypes.POINTER(CCmlTokens), vp, vp, vp, vp, vp]
+    lib.asynclm_token_monitor_step.argtypes = [vp, i32, i32, i32, i64, ctypes.POINTER(CCmlTokens), vp, vp, vp, vp, vp, vp]
+    lib.asynclm_token_monitor_workspace_bytes.argtypes = [i32]
     lib.asynclm_trap_decide.argtypes = [ctypes.POINTER(CTrapModel), i32, ctypes.c_double,
                                         ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_double),
                                         ctypes.POINTER(ctypes.c_double)]
@@ -131,10 +132,11 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_last_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     for name in EXPORTS:
         if name not in ("asynclm_strerror", "asynclm_last_cuda_error", "asynclm_static_scratch_bytes",
-                        "asynclm_kv_swap_staging_bytes"):
+                        "asynclm_kv_swap_staging_bytes", "asynclm_token_monitor_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     lib.asynclm_static_scratch_bytes.restype = ctypes.c_size_t
     lib.asynclm_kv_swap_staging_bytes.restype = ctypes.c_size_t
+    lib.asynclm_token_monitor_workspace_bytes.restype = ctypes.c_size_t
     _lib = lib
     return lib
 
@@ -318,16 +320,22 @@ def asynclm_trap_decide(model: dict, context_tokens: int, wait_us: float):
     return int(dec.value), float(s.value), float(r.value)
 
 
-def asynclm_token_monitor_step(logits, special: dict, state_in, token_out, state_out, flags_out, stream=None) -> None:
+def token_monitor_workspace_bytes(batch: int) -> int:
+    return int(load().asynclm_token_monitor_workspace_bytes(int(batch)))
+
+
+def asynclm_token_monitor_step(logits, special: dict, state_in, token_out, state_out, flags_out, workspace,
+                               stream=None) -> None:
     """Masked greedy next token and CML state advance for a batch (device tensors; logits bf16 or fp32,
-    [batch][vocab]); special: {"CALL", "INTR", "TRAP", "END", "HEAD"} -> token id."""
+    [batch][vocab]); special: {"CALL", "INTR", "TRAP", "END", "HEAD"} -> token id; workspace: zeroed
+    uint8 device tensor of token_monitor_workspace_bytes(batch) bytes (left zeroed)."""
     import torch
     ct = CCmlTokens(*(int(special[k]) for k in ("CALL", "INTR", "TRAP", "END", "HEAD")))
     dtype = 0 if logits.dtype == torch.bfloat16 else 1
     _check(load().asynclm_token_monitor_step(logits.data_ptr(), dtype, logits.shape[0], logits.shape[1],
                                              logits.stride(0), ctypes.byref(ct), state_in.data_ptr(),
                                              token_out.data_ptr(), state_out.data_ptr(), flags_out.data_ptr(),
-                                             _stream_ptr(stream)), "asynclm_token_monitor_step")
+                                             workspace.data_ptr(), _stream_ptr(stream)), "asynclm_token_monitor_step")
 
 
 def asynclm_latency_model(gen, exe) -> dict:

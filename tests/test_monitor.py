@@ -24,8 +24,13 @@ def run(logits_bits_or_f32, states, special, bf16):
     logits = full[:, :vocab]
     st = torch.from_numpy(np.asarray(states, dtype=np.int32)).cuda()
     tok, nxt, fl = (torch.full_like(st, -7) for _ in range(3))
-    B.asynclm_token_monitor_step(logits, special, st, tok, nxt, fl)
+    ws = torch.zeros(B.token_monitor_workspace_bytes(n), dtype=torch.uint8, device="cuda")
+    B.asynclm_token_monitor_step(logits, special, st, tok, nxt, fl, ws)
+    first = (tok.clone(), nxt.clone(), fl.clone())
+    tok.fill_(-7)
+    B.asynclm_token_monitor_step(logits, special, st, tok, nxt, fl, ws)      # the workspace came back zeroed
     torch.cuda.synchronize()
+    assert int(ws.max()) == 0 and all(torch.equal(a, b) for a, b in zip(first, (tok, nxt, fl)))
     return tok.cpu().numpy(), nxt.cpu().numpy(), fl.cpu().numpy()
 
 
