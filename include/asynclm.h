@@ -202,6 +202,18 @@ int asynclm_kv_append(const asynclm_plan_t* plan, const void* k_new, const void*
                       void* kv_pool, void* stream);
 
 /*
+ * asynclm_kv_append with the rotary position embedding fused in, as the layers of a Llama-family model
+ * (the models of the paper's evaluation, Section 6) need it: the key row of new token i of sequence b
+ * is rotated by its position ctx_b + i before it is stored (rotate-half pairs (j, j + d/2), angle
+ * position * rope_theta^(-2j / head_dim)), the value row is copied bit for bit, and, if q_inout is
+ * given, the step's query rows [T][num_q_heads][head_dim] are rotated in place by the same positions.
+ * Angles and products are evaluated in fp64 and rounded once to bf16.  Slots as in asynclm_kv_append.
+ * Errors: INVALID_ARG (also rope_theta <= 1), CUDA.
+ */
+int asynclm_kv_append_rope(const asynclm_plan_t* plan, const void* k_new, const void* v_new, void* kv_pool,
+                           void* q_inout, double rope_theta, void* stream);
+
+/*
  * Mixed decode + interrupt-append attention (Section 5.3: the appended tokens are processed in the
  * next decoding step, alongside the other sequences' single-token decodes).  Must follow
  * asynclm_kv_append on the same stream: the new rows are read back from the pages.  For every new

@@ -23,6 +23,7 @@ EXPORTS = [
     "asynclm_static_scratch_bytes", "asynclm_step", "asynclm_read_ceiling", "asynclm_kv_swap_staging_bytes",
     "asynclm_kv_swap_out", "asynclm_kv_swap_in", "asynclm_trap_decide", "asynclm_latency_model",
     "asynclm_async_latency_of_order", "asynclm_token_monitor_step", "asynclm_token_monitor_workspace_bytes",
+    "asynclm_kv_append_rope",
 ]
 
 TRAP_KEEP, TRAP_SWAP, TRAP_RECOMPUTE = 0, 1, 2
@@ -115,6 +116,7 @@ def load(rebuild_if_stale: bool = True):
     lib.asynclm_plan_get_items.argtypes = [vp, vp, i32]
     lib.asynclm_kv_append.argtypes = [vp, vp, vp, vp, vp]
     lib.asynclm_attn_mixed.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.asynclm_kv_append_rope.argtypes = [vp, vp, vp, vp, vp, ctypes.c_double, vp]
     lib.asynclm_attn_mixed_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.asynclm_step.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.asynclm_read_ceiling.argtypes = [vp, vp, i64, i64, i32, vp, vp]
@@ -273,6 +275,13 @@ def asynclm_kv_append(plan: Plan, k_new, v_new, kv_pool, stream=None) -> None:
     """Scatter the step's new K/V rows (device tensors) into kv_pool through the page table."""
     _check(load().asynclm_kv_append(plan.handle, k_new.data_ptr(), v_new.data_ptr(),
                                     kv_pool.data_ptr(), _stream_ptr(stream)), "asynclm_kv_append")
+
+
+def asynclm_kv_append_rope(plan: Plan, k_new, v_new, kv_pool, q_inout=None, rope_theta=500000.0, stream=None) -> None:
+    """asynclm_kv_append with the keys (and, if given, the queries, in place) rotated by their positions."""
+    _check(load().asynclm_kv_append_rope(plan.handle, k_new.data_ptr(), v_new.data_ptr(), kv_pool.data_ptr(),
+                                         None if q_inout is None else q_inout.data_ptr(), float(rope_theta),
+                                         _stream_ptr(stream)), "asynclm_kv_append_rope")
 
 
 def asynclm_attn_mixed(plan: Plan, q, kv_pool, out, lse=None, stream=None) -> None:
