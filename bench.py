@@ -646,6 +646,71 @@ def run_trap(args):
         "model": model, "decision_by_tokens_then_wait_us": table}))
 
 
+def run_layers(args):
+    """A whole decoding step's attention for a model of --layers layers with the Llama-3-8B attention
+    shape: one plan per step, then per layer the rotary append into that layer's pool and the mixed
+    attention over it (paper Section 4.2 quotes 5-30 ms per output token for whole models; this is the
+    attention part).  Every layer has a pool of its own (the default workload's), so a step streams
+    layers x 318 MB and nothing of a layer survives in L2 until the next step.  The step is also
+    replayed from a CUDA graph.  Prints one JSON line.  Not the benchmarked metric."""
+    import torch
+    from paper_2412_07017_b200 import binding as B
+    from paper_2412_07017_b200 import workload as W
+    torch.cuda.set_device(0)
+    L = args.layers
+    wl = W.make_config(2)
+    st, shape = wl.steps[0], wl.shape
+
+    def dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    pools = [dev(wl.kv_pool) for _ in range(L)]
+    q0, kn, vn = dev(st.q), dev(st.k_new), dev(st.v_new)
+    qs = [q0.clone() for _ in range(L)]
+    out = torch.empty_like(q0)
+    plan = B.asynclm_plan(shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices)
+    stream = torch.cuda.current_stream()
+
+    def step(s):
+        for l in range(L):
+            B.asynclm_kv_append_rope(plan, kn, vn, pools[l], qs[l], 500000.0, s)
+            B.asynclm_attn_mixed(plan, qs[l], pools[l], out, None, s)
+
+    def timed(fn, n):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(n)]
+        for k in range(n):
+            ev[k][0].record(torch.cuda.current_stream())
+            fn()
+            ev[k][1].record(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        return float(np.median([e[0].elapsed_time(e[1]) for e in ev])) * 1e3
+
+    for _ in range(3):
+        step(stream)
+    torch.cuda.synchronize()
+    eager_us = timed(lambda: step(stream), 20)
+    graph_us, graph_note = None, None
+    try:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step(torch.cuda.current_stream())
+        g.replay()
+        torch.cuda.synchronize()
+        graph_us = timed(g.replay, 20)
+    except Exception as e:      # capture is an extra; the eager number stands without it
+        graph_note = f"capture failed: {type(e).__name__}"
+    assert B.last_device_status(plan) == 0
+    peak, kind = measured_peaks()
+    by = W.algorithmic_bytes(shape, st)
+    best = min(x for x in (eager_us, graph_us) if x)
+    print(json.dumps({
+        "what": f"attention of one decoding step, {L} layers, Llama-3-8B attention shape, default mixed batch",
+        "layers": L, "us_per_step_eager": eager_us, "us_per_step_cuda_graph": graph_us, "graph_note": graph_note,
+        "us_per_layer": best / L, "kv_gbs": L * by["kv"] / best / 1e3,
+        "step_hbm_frac_of_" + kind: L * by["total"] / best / 1e3 / peak,
+        "launches_per_step": L * (1 + plan.info["launches_attn"])}))
+
+
 def run_monitor(args):
     """Token monitor (paper Section 5.1): masked greedy selection + CML state advance over bf16 logits of
     the Llama-3 vocabulary (128 256) for 256 sequences; bound by HBM (one read of the logits).  Prints one
@@ -701,10 +766,14 @@ def main():
                          "instead of benchmarking")
     ap.add_argument("--trap", action="store_true",
                     help="measure KV swap and attention recompute times and print the trap handler's cost model")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="time the attention of one decoding step of a model with this many layers instead")
     ap.add_argument("--monitor", action="store_true",
                     help="time the token monitor's masked selection kernel instead")
     args = ap.parse_args()
-    if args.monitor:
+    if args.layers > 0:
+        run_layers(args)
+    elif args.monitor:
         run_monitor(args)
     elif args.timeline:
         run_timeline(args)
