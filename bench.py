@@ -721,7 +721,8 @@ def run_monitor(args):
     batch, vocab = 256, 128256
     logits = torch.empty((batch, vocab), dtype=torch.bfloat16, device="cuda").normal_()
     special = {"CALL": 128011, "INTR": 128012, "TRAP": 128013, "END": 128014, "HEAD": 128015}
-    state = torch.from_numpy(np.random.default_rng(0).integers(0, 4, batch).astype(np.int32)).cuda()
+    # mostly plain text, some sequences inside a function-call block, a few right after [TRAP]
+    state = torch.from_numpy(np.random.default_rng(0).choice(4, batch, p=[0.8, 0.08, 0.1, 0.02]).astype(np.int32)).cuda()
     tok, nxt, fl = (torch.empty_like(state) for _ in range(3))
     ws = torch.zeros(B.token_monitor_workspace_bytes(batch), dtype=torch.uint8, device="cuda")
     flush = L2Flush(torch)

@@ -102,6 +102,39 @@ cudaError_t make_kv_map(const DevPlan& p, const void* pool, CUtensorMap* map) {
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device instead of once per launch.
+template <typename Kernel>
+cudaError_t allow_smem(Kernel kernel, size_t bytes) {
+    static std::atomic<unsigned long long> done{0};      // one per kernel instantiation; bit = device (first 64)
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = dev < 64 ? 1ull << dev : 0ull;
+    if (bit != 0 && (done.load(std::memory_order_acquire) & bit) != 0) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && bit != 0) done.fetch_or(bit, std::memory_order_release);
+    return e;
+}
+
+// The tensor map of a pool depends on its address and shape only: the last few are kept per thread.
+cudaError_t cached_kv_map(const DevPlan& p, const void* pool, CUtensorMap* map) {
+    struct Entry { const void* pool; int64_t pages; int hkv, d; CUtensorMap map; };
+    constexpr int kEntries = 8;
+    thread_local Entry cache[kEntries] = {};
+    thread_local int next = 0;
+    for (int i = 0; i < kEntries; ++i)
+        if (cache[i].pool == pool && cache[i].pages == p.num_pages && cache[i].hkv == p.num_kv_heads && cache[i].d == p.head_dim) {
+            *map = cache[i].map;
+            return cudaSuccess;
+        }
+    const cudaError_t e = make_kv_map(p, pool, map);
+    if (e == cudaSuccess) {
+        cache[next] = Entry{pool, p.num_pages, p.num_kv_heads, p.head_dim, *map};
+        next = (next + 1) % kEntries;
+    }
+    return e;
+}
+
 template <int D>
 int decode_stages() {
     int S = 6;
@@ -114,10 +147,10 @@ cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, voi
                           cudaStream_t stream, AppendSrc app) {
     const int S = decode_stages<D>();
     const size_t smem = dec::smem_bytes<D>(S);
-    cudaError_t e = cudaFuncSetAttribute(attn_decode_kernel<D, G, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_smem(attn_decode_kernel<D, G, APPEND>, smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
-    e = make_kv_map(p, pool, &map);
+    e = cached_kv_map(p, pool, &map);
     if (e != cudaSuccess) return e;
     return launch_pdl(attn_decode_kernel<D, G, APPEND>, dim3(p.num_ctas_cuda), dim3(dec::kThreads), smem, stream, p, map,
                       (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, S, app);
@@ -126,8 +159,7 @@ cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, voi
 template <int G, bool APPEND>
 cudaError_t launch_tensor(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                           cudaStream_t stream, AppendSrc app) {
-    cudaError_t e = cudaFuncSetAttribute(attn_append_tc_kernel<G, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)tc::kSmemBytes);
+    cudaError_t e = allow_smem(attn_append_tc_kernel<G, APPEND>, tc::kSmemBytes);
     if (e != cudaSuccess) return e;
     return launch_pdl(attn_append_tc_kernel<G, APPEND>, dim3(p.num_ctas_tensor), dim3(tc::kThreads), tc::kSmemBytes, stream,
                       p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, app);
@@ -138,10 +170,10 @@ cudaError_t launch_fused(const DevPlan& p, const void* q, const void* pool, void
                          cudaStream_t stream, AppendSrc app) {
     const int S = decode_stages<tc::kD>();
     const size_t smem = dec::smem_bytes<tc::kD>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD>(S) : tc::kSmemBytes;
-    cudaError_t e = cudaFuncSetAttribute(attn_fused_kernel<G, APPEND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_smem(attn_fused_kernel<G, APPEND>, smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
-    e = make_kv_map(p, pool, &map);
+    e = cached_kv_map(p, pool, &map);
     if (e != cudaSuccess) return e;
     return launch_pdl(attn_fused_kernel<G, APPEND>, dim3(p.num_ctas_cuda), dim3(tc::kThreads), smem, stream, p, map,
                       (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, S, app);

@@ -6,8 +6,8 @@
 // which interrupts are deferred, Section 3.2).
 //
 // The logits are streamed once (16-byte loads, several CTAs per sequence): the kernel is bound by HBM,
-// vocab * element size bytes per sequence.  The mask costs nothing per element: the five CML tokens are
-// set aside during the scan and compared at the end according to the state.
+// vocab * element size bytes per sequence.  The mask costs nothing per element: the scan takes the
+// plain maximum, and only a row whose maximum is a token its state forbids is looked at a second time.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -56,98 +56,174 @@ __device__ __forceinline__ Best unpack_key(unsigned long long k) {
     return Best{__uint_as_float(u), 0x7fffffff - (int)(unsigned)(k & 0xffffffffu)};
 }
 
-// Grid: (slices, batch).  Every CTA scans one slice of a sequence's row and folds its best ordinary
-// token into the row's key with one atomic max; the CTA that arrives last (per-row counter) finishes the
-// row: it lets the CML tokens the state allows compete, advances the state machine and puts the two
-// workspace words back to zero for the next call.  The result does not depend on arrival order.
+template <typename T> struct Vec;
+template <> struct Vec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    // largest of the 8 values of a 16-byte vector (NaN drops out of max)
+    static __device__ __forceinline__ float vmax(const uint4& w) {
+        const unsigned u[4] = {w.x, w.y, w.z, w.w};
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) m = fmaxf(m, fmaxf(bf16_lo(u[k]), bf16_hi(u[k])));
+        return m;
+    }
+    static __device__ __forceinline__ float at(const uint4& w, int k) {
+        const unsigned u[4] = {w.x, w.y, w.z, w.w};
+        return (k & 1) ? bf16_hi(u[k >> 1]) : bf16_lo(u[k >> 1]);
+    }
+};
+template <> struct Vec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ float vmax(const uint4& w) {
+        return fmaxf(fmaxf(__uint_as_float(w.x), __uint_as_float(w.y)), fmaxf(__uint_as_float(w.z), __uint_as_float(w.w)));
+    }
+    static __device__ __forceinline__ float at(const uint4& w, int k) {
+        const unsigned u[4] = {w.x, w.y, w.z, w.w};
+        return __uint_as_float(u[k]);
+    }
+};
+
+// Largest element of vectors [j_begin, j_end) of a row (stride of the CTA's threads), lowest id among
+// equals; `skip`: leave the five CML tokens out.  Per vector only its maximum is computed; the
+// position inside the best vector is found at the end by looking at that one vector again.
 template <typename T>
-__global__ void __launch_bounds__(kMonThreads)
-token_monitor_kernel(const T* __restrict__ logits, int vocab, int64_t row_stride, asynclm_cml_tokens tok,
-                     const int32_t* __restrict__ state_in, int32_t* __restrict__ token_out,
-                     int32_t* __restrict__ state_out, int32_t* __restrict__ flags_out,
-                     unsigned long long* __restrict__ ws) {
-    constexpr int VEC = 16 / sizeof(T);
-    const int seq = blockIdx.y;
-    const T* row = logits + (int64_t)seq * row_stride;
-    Best best{-INFINITY, INT_MAX};
-    auto offer = [&](float v, int i) {
-        // NaN fails both comparisons; the CML tokens take no part in the scan
-        if (better(v, i, best) && !is_special(i, tok)) best = Best{v, i};
-    };
-    const int nvec = vocab / VEC;
-    const int per = (nvec + gridDim.x - 1) / gridDim.x;
-    const int j_end = min(nvec, (int)(blockIdx.x + 1) * per);
-    for (int j0 = blockIdx.x * per + threadIdx.x; j0 < j_end; j0 += kMonVecs * kMonThreads) {
+__device__ __forceinline__ Best scan_row(const T* row, int j_begin, int j_end, const asynclm_cml_tokens& tok, bool skip) {
+    constexpr int VEC = Vec<T>::N;
+    const uint4* v4 = reinterpret_cast<const uint4*>(row);
+    float bv = -INFINITY;
+    int bj = -1;
+    for (int j0 = j_begin + threadIdx.x; j0 < j_end; j0 += kMonVecs * kMonThreads) {
         uint4 w[kMonVecs];
 #pragma unroll
         for (int u = 0; u < kMonVecs; ++u) {
             const int j = j0 + u * kMonThreads;
-            if (j < j_end) w[u] = ldg_nc_v4(reinterpret_cast<const uint4*>(row) + j);
+            if (j < j_end) w[u] = ldg_nc_v4(v4 + j);
         }
 #pragma unroll
         for (int u = 0; u < kMonVecs; ++u) {
             const int j = j0 + u * kMonThreads;
             if (j >= j_end) break;
-            const T* e = reinterpret_cast<const T*>(&w[u]);
-            // the vector's largest value first: only a vector that can change the best is looked at
-            // element by element (NaN compares false everywhere and drops out of fmaxf)
-            float vmax = -INFINITY;
+            float m = Vec<T>::vmax(w[u]);
+            if (skip) {      // (the rare second pass) recompute without the CML tokens this vector may hold
+                m = -INFINITY;
 #pragma unroll
-            for (int k = 0; k < VEC; ++k) vmax = fmaxf(vmax, to_f32<T>(e[k]));
-            if (vmax >= best.v) {
-                // (the five CML ids are tested per vector, not per element: a vector that holds none of
-                // them, which is nearly every vector, takes the short path)
-                const int lo = j * VEC;
-                const bool has_special = (unsigned)(tok.call - lo) < VEC || (unsigned)(tok.intr - lo) < VEC ||
-                                         (unsigned)(tok.trap - lo) < VEC || (unsigned)(tok.end - lo) < VEC ||
-                                         (unsigned)(tok.head - lo) < VEC;
-                if (has_special) {
-#pragma unroll
-                    for (int k = 0; k < VEC; ++k) offer(to_f32<T>(e[k]), lo + k);
-                } else {
-#pragma unroll
-                    for (int k = 0; k < VEC; ++k) {
-                        const float v = to_f32<T>(e[k]);
-                        if (better(v, lo + k, best)) best = Best{v, lo + k};
-                    }
-                }
+                for (int k = 0; k < VEC; ++k)
+                    if (!is_special(j * VEC + k, tok)) m = fmaxf(m, Vec<T>::at(w[u], k));
             }
+            if (m > bv) { bv = m; bj = j; }      // a thread's vectors come in increasing order: the first one wins a tie
         }
     }
-    if (blockIdx.x == gridDim.x - 1)
-        for (int i = nvec * VEC + threadIdx.x; i < vocab; i += kMonThreads) offer(to_f32<T>(row[i]), i);
-    // CTA-wide best: shuffles inside a warp, shared memory across warps
+    Best best{-INFINITY, INT_MAX};
+    if (bj >= 0) {
+        const uint4 w = ldg_nc_v4(v4 + bj);
+#pragma unroll
+        for (int k = VEC - 1; k >= 0; --k)
+            if (Vec<T>::at(w, k) == bv && !(skip && is_special(bj * VEC + k, tok))) best = Best{bv, bj * VEC + k};
+    }
+    return best;
+}
+
+// CTA-wide best in thread 0 (shuffles inside a warp, shared memory across warps).
+__device__ __forceinline__ Best block_best(Best best, float* sv, int* si) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         const float v = __shfl_xor_sync(0xffffffffu, best.v, off);
         const int i = __shfl_xor_sync(0xffffffffu, best.i, off);
         if (better(v, i, best)) best = Best{v, i};
     }
-    __shared__ float sv[kMonThreads / 32];
-    __shared__ int si[kMonThreads / 32];
+    __syncthreads();      // (sv / si may still be read from an earlier call)
     if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best.v; si[threadIdx.x >> 5] = best.i; }
     __syncthreads();
-    if (threadIdx.x != 0) return;
-    for (int w = 1; w < kMonThreads / 32; ++w)
-        if (better(sv[w], si[w], best)) best = Best{sv[w], si[w]};
+    if (threadIdx.x == 0)
+        for (int w = 1; w < kMonThreads / 32; ++w)
+            if (better(sv[w], si[w], best)) best = Best{sv[w], si[w]};
+    return best;
+}
+
+// Grid: (slices, batch).  Every CTA scans one slice of a sequence's row, ALL tokens alike, and folds its
+// best into the row's key with one atomic max; the CTA that arrives last (per-row counter) finishes the
+// row.  If the row's largest logit belongs to an ordinary token or to a CML token the state allows, that
+// token is the answer (an allowed token that beats everything beats everything allowed).  Only if it
+// belongs to a CML token the state forbids, a "hallucinated" [INTR] say, the last CTA scans the row once
+// more without the CML tokens and lets the allowed ones compete.  Then the state machine advances and
+// the two workspace words go back to zero.  The result does not depend on arrival order.
+template <typename T>
+__global__ void __launch_bounds__(kMonThreads)
+token_monitor_kernel(const T* __restrict__ logits, int vocab, int64_t row_stride, asynclm_cml_tokens tok,
+                     const int32_t* __restrict__ state_in, int32_t* __restrict__ token_out,
+                     int32_t* __restrict__ state_out, int32_t* __restrict__ flags_out,
+                     unsigned long long* __restrict__ ws) {
+    constexpr int VEC = Vec<T>::N;
+    __shared__ float sv[kMonThreads / 32];
+    __shared__ int si[kMonThreads / 32];
+    __shared__ int s_rescan;
+    const int seq = blockIdx.y;
+    const T* row = logits + (int64_t)seq * row_stride;
+    if (state_in[seq] == kTrap) {
+        // [TRAP] is followed by [END] whatever the logits say: nothing to read
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            token_out[seq] = tok.end;
+            state_out[seq] = kText;
+            flags_out[seq] = ASYNCLM_MONITOR_TRAP;
+        }
+        return;
+    }
+    const int nvec = vocab / VEC;
+    const int per = (nvec + gridDim.x - 1) / gridDim.x;
+    Best best = scan_row<T>(row, blockIdx.x * per, min(nvec, (int)(blockIdx.x + 1) * per), tok, false);
+    if (blockIdx.x == gridDim.x - 1)      // the row's ragged end, element by element
+        for (int i = nvec * VEC + threadIdx.x; i < vocab; i += kMonThreads) {
+            const float v = to_f32<T>(row[i]);
+            if (better(v, i, best)) best = Best{v, i};
+        }
+    best = block_best(best, sv, si);
     unsigned long long* key = ws + 2 * (size_t)seq;
     unsigned* arrived = reinterpret_cast<unsigned*>(key + 1);
-    if (best.i != INT_MAX) atomicMax(key, pack_key(best.v, best.i));
-    __threadfence();
-    if (atomicAdd(arrived, 1u) != gridDim.x - 1) return;
-    __threadfence();
-    best = unpack_key(atomicExch(key, 0ull));
-    *arrived = 0;
-    // ---- the state machine: which of the CML tokens compete, and where the chosen token leads
     const int state = state_in[seq];
-    Best pick = state == kTrap ? Best{-INFINITY, INT_MAX} : best;      // ordinary tokens: everywhere but in a trap block
-    auto compete = [&](int id) {
-        const float v = to_f32<T>(row[id]);
-        if (better(v, id, pick)) pick = Best{v, id};
+    auto allowed_special = [&](int id) {
+        return (state == kText && (id == tok.call || id == tok.trap)) || (state == kCall && (id == tok.head || id == tok.end)) ||
+               ((state == kBody || state == kTrap) && id == tok.end);
     };
-    if (state == kText) { compete(tok.call); compete(tok.trap); }
-    if (state == kCall) { compete(tok.head); compete(tok.end); }
-    if (state == kBody || state == kTrap) compete(tok.end);
+    if (threadIdx.x == 0) {
+        s_rescan = -1;      // -1: this CTA is not the last one of its row
+        if (best.i != INT_MAX) atomicMax(key, pack_key(best.v, best.i));
+        __threadfence();
+        if (atomicAdd(arrived, 1u) == gridDim.x - 1) {
+            __threadfence();
+            best = unpack_key(atomicExch(key, 0ull));
+            *arrived = 0;
+            const bool ordinary = best.i != INT_MAX && !is_special(best.i, tok);
+            // ordinary tokens are allowed everywhere but in a trap block
+            const bool settled = best.i != INT_MAX && best.v > -INFINITY &&
+                                 (ordinary ? state != kTrap : allowed_special(best.i));
+            s_rescan = settled ? 0 : 1;
+        }
+    }
+    __syncthreads();
+    if (s_rescan < 0) return;
+    if (s_rescan == 1) {
+        // the row's best ordinary token (none in a trap block), then the CML tokens the state allows
+        Best ord{-INFINITY, INT_MAX};
+        if (state != kTrap) {
+            ord = scan_row<T>(row, 0, nvec, tok, true);
+            for (int i = nvec * VEC + threadIdx.x; i < vocab; i += kMonThreads) {
+                const float v = to_f32<T>(row[i]);
+                if (!is_special(i, tok) && better(v, i, ord)) ord = Best{v, i};
+            }
+        }
+        ord = block_best(ord, sv, si);
+        if (threadIdx.x == 0) {
+            best = ord;
+            const int ids[5] = {tok.call, tok.trap, tok.head, tok.end, tok.intr};
+            for (int a = 0; a < 5; ++a)
+                if (allowed_special(ids[a])) {
+                    const float v = to_f32<T>(row[ids[a]]);
+                    if (better(v, ids[a], best)) best = Best{v, ids[a]};
+                }
+        }
+    }
+    if (threadIdx.x != 0) return;
+    Best pick = best;
     if (pick.i == INT_MAX || pick.v == -INFINITY) {
         // no allowed token has a logit above -inf (all NaN or -inf): the lowest allowed id is taken
         int low = 0;
