@@ -186,6 +186,25 @@ def run_reference(args):
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 
+def max_over_ranks(x: float) -> float:
+    """The largest of the ranks' values (the step time of the slowest replica); identity without a
+    process group.  Works on whichever backend the group has (NCCL on GPUs, gloo in the CPU tests)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([float(x)], device=dev, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(kv_bytes_per_replica: int, world: int, ms_per_step: float) -> float:
+    """GB/s of the whole job: every rank runs the same step on its own GPU (no exchange between them),
+    and the job's step takes as long as its slowest replica's."""
+    return world * kv_bytes_per_replica / (ms_per_step * 1e-3) / 1e9
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -283,10 +302,7 @@ def run_gpu(args):
         dist.barrier()
     step_ms = all_blocks[int(np.argsort([b.sum() for b in all_blocks])[len(all_blocks) // 2])]
     total_ms = float(step_ms.sum())
-    if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(total_ms)
     # Pass 2 (roofline of the dominant kernel): the same steps with one more event between the two
     # calls, which gives the duration of asynclm_attn_mixed alone (and serialises it behind the append).
     ev2 = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
@@ -385,10 +401,7 @@ def run_gpu(args):
         t0 = time.perf_counter()
         e2e_step()
         e2e_total += time.perf_counter() - t0
-    if world > 1:
-        tt = torch.tensor([e2e_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_total = float(tt.item())
+    e2e_total = max_over_ranks(e2e_total)
     h2d = in_h.numel() * 2      # + the plan upload (tens of KB)
     d2h = out_h.numel() * 2
 
@@ -399,7 +412,7 @@ def run_gpu(args):
 
     peak, peak_kind = measured_peaks()
     ms_per_step = total_ms / args.steps
-    value = world * by["kv"] / (ms_per_step * 1e-3) / 1e9
+    value = replica_throughput(by["kv"], world, ms_per_step)
     attn_bytes = by["kv"] + by["qo"] + by["page_ids"]
     attn_s = float(attn_ms.mean()) * 1e-3
     achieved = attn_bytes / attn_s / 1e9
