@@ -103,8 +103,10 @@ cudaError_t make_kv_map(const DevPlan& p, const void* pool, CUtensorMap* map) {
 }
 
 // cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device instead of once per launch.
-template <typename Kernel>
-cudaError_t allow_smem(Kernel kernel, size_t bytes) {
+// The kernel is a template VALUE: kernels of one signature share a pointer type, and a flag per type
+// would let the first of them stand for all.
+template <auto kernel>
+cudaError_t allow_smem(size_t bytes) {
     static std::atomic<unsigned long long> done{0};      // one per kernel instantiation; bit = device (first 64)
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -147,7 +149,7 @@ cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, voi
                           cudaStream_t stream, AppendSrc app) {
     const int S = decode_stages<D>();
     const size_t smem = dec::smem_bytes<D>(S);
-    cudaError_t e = allow_smem(attn_decode_kernel<D, G, APPEND>, smem);
+    cudaError_t e = allow_smem<attn_decode_kernel<D, G, APPEND>>(smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
     e = cached_kv_map(p, pool, &map);
@@ -159,7 +161,7 @@ cudaError_t launch_decode(const DevPlan& p, const void* q, const void* pool, voi
 template <int G, bool APPEND>
 cudaError_t launch_tensor(const DevPlan& p, const void* q, const void* pool, void* out, float* lse,
                           cudaStream_t stream, AppendSrc app) {
-    cudaError_t e = allow_smem(attn_append_tc_kernel<G, APPEND>, tc::kSmemBytes);
+    cudaError_t e = allow_smem<attn_append_tc_kernel<G, APPEND>>(tc::kSmemBytes);
     if (e != cudaSuccess) return e;
     return launch_pdl(attn_append_tc_kernel<G, APPEND>, dim3(p.num_ctas_tensor), dim3(tc::kThreads), tc::kSmemBytes, stream,
                       p, (const __nv_bfloat16*)q, (const __nv_bfloat16*)pool, (__nv_bfloat16*)out, lse, app);
@@ -170,7 +172,7 @@ cudaError_t launch_fused(const DevPlan& p, const void* q, const void* pool, void
                          cudaStream_t stream, AppendSrc app) {
     const int S = decode_stages<tc::kD>();
     const size_t smem = dec::smem_bytes<tc::kD>(S) > tc::kSmemBytes ? dec::smem_bytes<tc::kD>(S) : tc::kSmemBytes;
-    cudaError_t e = allow_smem(attn_fused_kernel<G, APPEND>, smem);
+    cudaError_t e = allow_smem<attn_fused_kernel<G, APPEND>>(smem);
     if (e != cudaSuccess) return e;
     CUtensorMap map;
     e = cached_kv_map(p, pool, &map);
