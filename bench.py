@@ -566,7 +566,11 @@ def run_timeline(args):
     from paper_2412_07017_b200 import binding as B
     from paper_2412_07017_b200 import workload as W
     torch.cuda.set_device(0)
-    wl = W.make_config(args.config)
+    if args.spans_only:
+        lens = np.random.default_rng(4).integers(1024, 3073, 24).tolist()
+        wl = W.make_single_step("spans-only", W.Shape(32, 8, 128, 16), lens, [64] * 24, seed=12)
+    else:
+        wl = W.make_config(args.config)
     st, shape = wl.steps[0], wl.shape
 
     def dev(bits):
@@ -576,21 +580,21 @@ def run_timeline(args):
     out = torch.empty((st.total_q, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
     plan = B.asynclm_plan(shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices)
     flush = L2Flush(torch)
-    buf = np.zeros((1024, 8), dtype=np.uint64)
+    buf = np.zeros((1024, 16), dtype=np.uint64)
     for k in range(6):
         flush.fill_(k)
         B.asynclm_kv_append(plan, kn, vn, pool)
         B.asynclm_attn_mixed(plan, q, pool, out, None)
         torch.cuda.synchronize()
         assert B.load().asynclm_trace_read(ctypes.c_void_p(buf.ctypes.data)) == 0
-    n = plan.info["num_ctas_cuda"]
+    n = plan.info["num_ctas_tensor"] if args.spans_only else plan.info["num_ctas_cuda"]
     t = buf[:n].astype(np.int64)
     t0 = t[:, 0].min()
     us = lambda col: (t[:, col] - t0) / 1e3
     span = t[:, 1] > 0
     stats = lambda a: [round(float(x), 1) for x in (a.min(), a.mean(), a.max())] if len(a) else None
     print(json.dumps({
-        "workload": WORKLOADS.get(args.config, str(args.config)), "ctas": int(n), "span_ctas": int(span.sum()),
+        "workload": "spans-only-24x[1024,3072]+64" if args.spans_only else WORKLOADS.get(args.config, str(args.config)), "ctas": int(n), "span_ctas": int(span.sum()),
         "entry_us_min_mean_max": stats(us(0)),
         "span_body_done_us_min_mean_max": stats(us(1)[span]),
         "first_page_copy_us_mean_ctas_without_span_work": round(float(us(2)[~span].mean()), 1) if (~span).any() else None,
@@ -599,6 +603,18 @@ def run_timeline(args):
         "warp_body_items_per_cta_mean": round(float(t[:, 5].mean()), 1),
         "warp_body_stages_per_cta_mean": round(float(t[:, 6].mean()), 1),
         "split_units_merged_per_cta_mean_max": [round(float(t[:, 7].mean()), 2), int(t[:, 7].max())],
+        # span body, SM cycles summed over a CTA's span tiles (CTAs with span work only)
+        "span_body_cycles_mean": None if not span.any() else {
+            "mma_thread_waits_for_P": round(float(t[span, 8].mean())),
+            "mma_thread_waits_for_KV": round(float(t[span, 9].mean())),
+            "mma_thread_item_loop": round(float(t[span, 10].mean())),
+            "group0_waits_for_S": round(float(t[span, 11].mean())),
+            "group1_waits_for_S": round(float(t[span, 15].mean())),
+            "group0_softmax_of_tiles": round(float(t[span, 12].mean())),
+            "group0_tiles": round(float(t[span, 13].mean()), 1),
+            "mma_thread_waits_for_item_start": round(float(t[span, 14].mean())),
+            "mma_thread_issues_QK (tensor-only kernel)": round(float(t[span, 2].mean())) if args.spans_only else None,
+            "mma_thread_issues_PV (tensor-only kernel)": round(float(t[span, 3].mean())) if args.spans_only else None},
         "plan": {k: plan.info[k] for k in ("num_items", "num_items_tensor", "num_split_units")}}))
 
 

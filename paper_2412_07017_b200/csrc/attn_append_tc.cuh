@@ -119,6 +119,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
+// The same wait without the back-off, for the one thread that issues the MMAs: what it waits for is on
+// the critical path of both softmax groups.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* status, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+    return true;
+}
 // The same wait with a warp-uniform verdict, for code that goes on to warp-collective instructions.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                int32_t* status, int code) {
@@ -408,71 +424,93 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             int item_no = 0;
             const uint32_t idesc_pv = instr_desc(128, 1);
             TItem it_next = load_titem(head_work, i0 < i1);
+            const long long t_loop = trace_clock();
+            long long tr_p = 0, tr_kv = 0, tr_item = 0, tr_qk = 0, tr_pv = 0;      // time-stamp build: cycles waiting for P, for K/V, for an item's Q and O
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
                 it_next = load_titem(p.works + ii + 1, ii + 1 < i1);      // in flight while this item runs
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
                 const bool dual = it.ntok * G > kTile;
-                ok = mbar_wait(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
+                const long long t_item = trace_clock();
+                ok = mbar_wait_spin(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
                 // S and O of the previous item are in use until its epilogue is over
-                if (ok && item_no > 0) ok = mbar_wait(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 27);
+                if (ok && item_no > 0) ok = mbar_wait_spin(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 27);
+                tr_item += trace_clock() - t_item;
                 if (ok) tc_fence_after();
                 auto tile_pages = [&](int j) { return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage; };
-                // S[b] <- Q[qt] K_j^T; release_k: this is the last use of the K tile
-                auto issue_qk = [&](int j, int b, bool release_k) {
+                // S[b] <- Q[qt] K_j^T, then one commit: it tells group b that S[b] is complete and, because MMAs
+                // complete in issue order, that every MMA in front of it is done as well (the group releases
+                // the ring slots on that knowledge: a second commit per batch costs the tensor pipe ~90 cycles)
+                auto issue_qk = [&](int j, int b) {
                     const int pos = ring_pos_k(gt + j), s = pos % kRing;
-                    ok = mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
+                    const long long tw = trace_clock();
+                    ok = mbar_wait_spin(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
+                    const long long ti = trace_clock();
+                    tr_kv += ti - tw;
                     if (!ok) return;
                     tc_fence_after();
                     const uint32_t idesc = instr_desc(16u * (uint32_t)tile_pages(j), 0);
                     const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
-                    const uint32_t qbase = sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u);
-                    const uint32_t kbase = sbase + kOffRing + s * kTileBytes;
+                    const uint64_t qd = smem_desc(sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u), 16, 1024);
+                    const uint64_t kd = smem_desc(sbase + kOffRing + s * kTileBytes, 16, 1024);
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks) {
-                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        mma_f16(d, smem_desc(qbase + off, 16, 1024), smem_desc(kbase + off, 16, 1024), idesc, ks > 0);
+                        // the address field counts 16-byte units and cannot carry out of its 14 bits here
+                        const uint64_t off = (uint64_t)(((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4);
+                        mma_f16(d, qd + off, kd + off, idesc, ks > 0);
                     }
                     mma_commit(bar(kSFull0 + 2 * b));
-                    if (release_k) mma_commit(bar(kRingEmpty0 + s));
+                    tr_qk += trace_clock() - ti;
                 };
-                // O[b] (+)= P[b] V_j with P[b] in tensor memory; fresh: first P V of the item into O[b]
-                auto issue_pv = [&](int j, int b, bool fresh, bool release_v) {
+                // O[b] (+)= P[b] V_j with P[b] in tensor memory; fresh: first P V of the item into O[b];
+                // last: the group's last tile of the item, the only one whose completion is signalled by itself
+                auto issue_pv = [&](int j, int b, bool fresh, bool last) {
                     const int pos = ring_pos_v(gt + j), s = pos % kRing;
-                    ok = mbar_wait(bar(kPFull0 + 2 * b), (uint32_t)(b ? cnt1 : cnt0) & 1u, abort_flag, p.status, 26) &&
-                         mbar_wait(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
+                    const long long tw = trace_clock();
+                    ok = mbar_wait_spin(bar(kPFull0 + 2 * b), (uint32_t)(b ? cnt1 : cnt0) & 1u, abort_flag, p.status, 26);
+                    const long long tv = trace_clock();
+                    tr_p += tv - tw;
+                    ok = ok && mbar_wait_spin(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
+                    const long long ti = trace_clock();
+                    tr_kv += ti - tv;
                     if (!ok) return;
                     tc_fence_after();
                     const int npg = tile_pages(j);
                     const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b;
+                    const uint64_t vd = smem_desc(sbase + kOffRing + s * kTileBytes, kHalfBytes, 1024);
                     for (int ks = 0; ks < npg; ++ks)
-                        mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks,
-                                   smem_desc(sbase + kOffRing + s * kTileBytes + (uint32_t)ks * 2 * 1024u, kHalfBytes, 1024),
+                        mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks, vd + (uint64_t)(ks * 128),
                                    idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
-                    mma_commit(bar(kPvDone0 + 2 * b));
+                    if (last) mma_commit(bar(kPvDone0 + 2 * b));
                     if (b) ++cnt1; else ++cnt0;
-                    if (release_v) mma_commit(bar(kRingEmpty0 + s));
+                    tr_pv += trace_clock() - ti;
                 };
                 if (dual) {
                     // both groups on every tile: group b owns row tile b
-                    if (ok) issue_qk(0, 0, false);
-                    if (ok) issue_qk(0, 1, true);
+                    if (ok) issue_qk(0, 0);
+                    if (ok) issue_qk(0, 1);
                     for (int j = 0; j < ntiles && ok; ++j)
                         for (int b = 0; b < 2 && ok; ++b) {
-                            issue_pv(j, b, j == 0, b == 1);
-                            if (ok && j + 1 < ntiles) issue_qk(j + 1, b, b == 1);
+                            issue_pv(j, b, j == 0, j + 1 == ntiles);
+                            if (ok && j + 1 < ntiles) issue_qk(j + 1, b);
                         }
                 } else {
                     // one row tile: the groups take alternate KV tiles
-                    if (ok) issue_qk(0, 0, true);
-                    if (ok && ntiles > 1) issue_qk(1, 1, true);
+                    if (ok) issue_qk(0, 0);
+                    if (ok && ntiles > 1) issue_qk(1, 1);
                     for (int j = 0; j < ntiles && ok; ++j) {
-                        issue_pv(j, j & 1, j < 2, true);
-                        if (ok && j + 2 < ntiles) issue_qk(j + 2, j & 1, true);
+                        issue_pv(j, j & 1, j < 2, j + 2 >= ntiles);
+                        if (ok && j + 2 < ntiles) issue_qk(j + 2, j & 1);
                     }
                 }
                 gt += ntiles;
             }
+            trace_set(8, tr_p);
+            trace_set(9, tr_kv);
+            trace_set(10, trace_clock() - t_loop);
+            trace_set(14, tr_item);
+            trace_set(2, tr_qk);
+            trace_set(3, tr_pv);
             // make sure nothing is still running on the tensor core before tensor memory is released
             mma_commit(bar(kMmaDrain));
             const long long t0 = clock64();
@@ -490,8 +528,11 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         const float qscale = p.sm_scale * kLog2e;
         const float2 qscale2 = make_float2(qscale, qscale);
         int cnt = 0;         // tiles this group has processed before this item
+        int gt = 0;          // KV tiles of the CTA before this item (both groups): ring position
+        int pv_cnt = 0;      // items so far in which this group had tiles: phase of its "last P V done" barrier
         int item_no = 0;
         bool ok = true;
+        long long tr_wait = 0, tr_work = 0, tr_tiles = 0;      // time-stamp build: cycles waiting for S, cycles from S to P, tiles
         // This thread's share of an item's Q.  Dual items: the whole row 128 b + m (16 chunks of 16
         // bytes) into Q[b]; otherwise value half b of row m (8 chunks) into Q[0].  The next item's Q is
         // fetched at the end of the current item's KV loop, ahead of the epilogue.
@@ -544,9 +585,20 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 const int npg = (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage;
                 // S[b] complete; it was issued after the P V of this group's previous tile finished, so
                 // O[b] is at rest as well
+                const long long tw = trace_clock();
                 ok = mbar_wait_warp(bar(kSFull0 + 2 * b), (uint32_t)(cnt + mine) & 1u, abort_flag, p.status, 31);
+                const long long ts = trace_clock();
+                tr_wait += ts - tw;
+                ++tr_tiles;
                 if (!ok) break;
                 tc_fence_after();
+                // S[b] of tile j complete means every MMA issued before it is complete.  The group that is
+                // last to use a ring slot gives it back to the producers: the K tile of j now, and the V tile
+                // of the group's previous tile (its P V was issued in front of this Q K^T).
+                if (m == 0 && (!dual || b == 1)) {
+                    mbar_arrive(bar(kRingEmpty0 + ring_pos_k(gt + j) % kRing));
+                    if (mine > 0) mbar_arrive(bar(kRingEmpty0 + ring_pos_v(gt + j - (dual ? 1 : 2)) % kRing));
+                }
                 // the tile is handled in two halves of 64 keys (register budget)
                 for (int h = 0; h * 4 < npg; ++h) {
                     const int base = it.kv0 + j * kTile + h * kSub;
@@ -640,6 +692,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(kPFull0 + 2 * b));
+                tr_work += trace_clock() - ts;
             }
             if (!ok) break;
             const float l_sum = (l2.x + l2.y) + (l2b.x + l2b.y);
@@ -647,9 +700,13 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             // ---- epilogue.  The groups' (max, sum) go through columns 0-1 of their S buffers, which are
             // idle from the group's last P V until the next item's first Q K^T.
             if (mine > 0) {
-                ok = mbar_wait_warp(bar(kPvDone0 + 2 * b), (uint32_t)(cnt + mine - 1) & 1u, abort_flag, p.status, 34);
+                ok = mbar_wait_warp(bar(kPvDone0 + 2 * b), (uint32_t)pv_cnt & 1u, abort_flag, p.status, 34);
                 if (!ok) break;
+                ++pv_cnt;
                 tc_fence_after();
+                // the V tile of the group's last tile goes back to the producers
+                if (m == 0 && (!dual || b == 1))
+                    mbar_arrive(bar(kRingEmpty0 + ring_pos_v(gt + (dual ? ntiles - 1 : b + 2 * (mine - 1))) % kRing));
             }
             tmem_st2(s_addr, __float_as_uint(m_ref), __float_as_uint(l_sum));
             tmem_wait_st();
@@ -761,6 +818,11 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             tc_fence_before();
             mbar_arrive(bar(kOFree));
             cnt += mine;
+            gt += ntiles;
+        }
+        if ((threadIdx.x & 127) == 0) {
+            trace_set(b ? 15 : 11, tr_wait);
+            if (b == 0) { trace_set(12, tr_work); trace_set(13, tr_tiles); }
         }
     }
 

@@ -42,7 +42,12 @@ attn_append_tc_kernel(DevPlan p, const __nv_bfloat16* __restrict__ q, const __nv
                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse, AppendSrc app) {
     extern __shared__ uint8_t smem_raw[];
     pdl_trigger();      // the kernel behind this one may start its prologue; it waits for this grid to complete
+    if (threadIdx.x == 0) {
+        trace_mark(0);
+        for (int s = 8; s < 16; ++s) trace_set(s, 0);
+    }
     tc::tc_body<G, APPEND>(p, q, pool, out, lse, aligned_smem(smem_raw), app);
+    if (threadIdx.x == 0) trace_mark(1);
 }
 
 template <int G, bool APPEND>
@@ -63,6 +68,9 @@ attn_fused_kernel(DevPlan p, const __grid_constant__ CUtensorMap kv_map, const _
         // no span tiles for this CTA: straight to its decode rows, without the tensor-memory set-up
         dec::decode_body<tc::kD, G, APPEND>(p, &kv_map, q, out, lse, S, smem, app);
         return;
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 8; s < 16; ++s) trace_set(s, 0);
     }
     tc::tc_body<G, APPEND>(p, q, pool, out, lse, smem, app);
     if (threadIdx.x == 0) trace_mark(1);

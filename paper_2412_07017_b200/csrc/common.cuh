@@ -61,7 +61,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // Per-CTA time stamps for performance work: compiled in only with -DASYNCLM_TRACE (see build.py),
 // read back with asynclm_trace_read().  Slot meanings are the callers'.
 #ifdef ASYNCLM_TRACE
-constexpr int kTraceSlots = 8, kTraceCtas = 1024;
+constexpr int kTraceSlots = 16, kTraceCtas = 1024;
 static __device__ unsigned long long g_trace[kTraceCtas][kTraceSlots];      // one copy per translation unit
 __device__ __forceinline__ void trace_mark(int slot) {
     unsigned long long t;
@@ -74,7 +74,9 @@ __device__ __forceinline__ void trace_add(int slot, unsigned long long v) {
 __device__ __forceinline__ void trace_set(int slot, unsigned long long v) {
     if (blockIdx.x < kTraceCtas) g_trace[blockIdx.x][slot] = v;
 }
+__device__ __forceinline__ long long trace_clock() { return clock64(); }
 #else
+__device__ __forceinline__ long long trace_clock() { return 0; }
 __device__ __forceinline__ void trace_mark(int) {}
 __device__ __forceinline__ void trace_add(int, unsigned long long) {}
 __device__ __forceinline__ void trace_set(int, unsigned long long) {}
