@@ -55,6 +55,11 @@ constexpr int kProducerWarpK = 8, kMmaWarp = 9, kProducerWarpV = 10, kAppendWarp
 constexpr int kD = 128;
 constexpr int kTile = 128;                       // keys per K/V ring slot and query rows per row tile
 constexpr int kSub = 64;                         // keys the softmax handles at a time (half an S tile)
+// Pairs (of the 16 of a quarter) whose exponentials are evaluated by polynomial instead of ex2.approx.
+#ifndef ASYNCLM_POLY_MASK
+#define ASYNCLM_POLY_MASK 0x4924u
+#endif
+constexpr uint32_t kPolyMask = ASYNCLM_POLY_MASK;
 constexpr int kRing = 5;                         // K/V ring slots
 constexpr uint32_t kHalfBytes = 128 * 128;       // one 64-value half of a 128-row tile
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;  // 32 KiB
@@ -169,6 +174,12 @@ __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\tselp.u32 %0, 1, 0, e;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -198,6 +209,16 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
         "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
         ::TC_W32(r), "r"(taddr) : "memory");
+}
+// Waits for this thread's tensor-memory loads; the loaded registers pass through the statement so that
+// no use of them can be scheduled in front of it.
+__device__ __forceinline__ void tmem_wait_ld_dep(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :: "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -232,6 +253,22 @@ __device__ __forceinline__ void mma_f16_ta(uint32_t d_tmem, uint32_t a_tmem, uin
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+
+// 2^x for two finite values on the FMA pipe: n = round(x) through the 1.5 * 2^23 trick, a cubic for
+// 2^(x - n) on [-1/2, 1/2] (relative error 7.5e-5, below the bf16 rounding of P), n added to the
+// exponent field.  x is clamped at -125 so that the exponent cannot wrap.
+__device__ __forceinline__ float2 poly_exp2(float2 x) {
+    const float kMagic = 12582912.f;
+    const float2 xc = make_float2(fmaxf(x.x, -125.f), fmaxf(x.y, -125.f));
+    const float2 t = __fadd2_rn(xc, make_float2(kMagic, kMagic));
+    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), xc);
+    float2 r = __ffma2_rn(f, make_float2(0.0551716685f, 0.0551716685f), make_float2(0.2426111251f, 0.2426111251f));
+    r = __ffma2_rn(r, f, make_float2(0.6932609677f, 0.6932609677f));
+    r = __ffma2_rn(r, f, make_float2(0.9999280572f, 0.9999280572f));
+    return make_float2(__int_as_float(__float_as_int(r.x) + (__float_as_int(t.x) << 23)),
+                       __int_as_float(__float_as_int(r.y) + (__float_as_int(t.y) << 23)));
 }
 
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
@@ -284,7 +321,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         mbar_init(bar(kStats), 256);
         mbar_init(bar(kOFree), 256);
         for (int b = 0; b < 4; ++b) {
-            mbar_init(bar(kPFull0 + b), 128);
+            mbar_init(bar(kPFull0 + b), 4);      // one arrival per warp of the group
             mbar_init(bar(kPvDone0 + b), 1);
             mbar_init(bar(kSFull0 + b), 1);
         }
@@ -320,6 +357,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         bool ok = true;
         int n = 0;                                             // KV tiles issued so far (all items)
         int last_pos = -1;
+        int ev = 0;      // time-stamp build: event log position (lane 0 of a producer)
         TItem cur = load_titem(head_work, i0 < i1), nxt = load_titem(p.works + i0 + 1, i0 + 1 < i1);
         int pages_cur = head[kHeadPagesTensor + lane];      // the first item's first 32 page ids (0 beyond its end)
         pdl_wait();
@@ -360,8 +398,10 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     }
                     const int pos = which ? ring_pos_v(n) : ring_pos_k(n);
                     const int s = pos % kRing;
+                    if (lane == 0) trace_event(9 + which, ev, 40);
                     ok = mbar_wait_warp(bar(kRingEmpty0 + s), ((uint32_t)(pos / kRing) & 1u) ^ 1u, abort_flag, p.status, 11 + which);
                     if (!ok) break;
+                    if (lane == 0) trace_event(9 + which, ev, 42);
                     last_pos = pos;
                     // lane -> 16-byte chunk c of row 2*rr + (lane >> 4) of each page: a warp instruction
                     // moves two whole 256-byte rows
@@ -380,6 +420,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                         }
                     }
                     cp_async_arrive(bar(kRingFull0 + s));
+                    if (lane == 0) trace_event(9 + which, ev, 44);
                     // page ids of the next group of tiles (or of the next item), requested only after this
                     // group's first tile is on its way: the next item's descriptor may still be in flight
                     if (t == t0) {
@@ -410,14 +451,16 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         }
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
-        // One thread issues every MMA of the CTA, in an order that lets the two softmax groups work
+        // One warp, running convergently, issues every MMA of the CTA through an elected lane (operands then
+        // stay in uniform registers: under a lane-0 branch each MMA took the lone thread 85-110 cycles to
+        // issue, against 64 cycles on the tensor core), in an order that lets the two softmax groups work
         // in turns: after the P V of a group's tile it issues the Q K^T of the same group's next tile
         // at once (MMAs of one thread execute in issue order, so the new S may overwrite the P that the
         // P V in front of it reads), then it turns to the other group.  While the tensor core works
         // for one group, the other group's softmax has the exponential unit to itself.
-        // An MMA costs about 94 cycles however narrow it is (measured), so Q K^T is issued 128 keys
-        // wide: 8 instructions per tile and group.
-        if (lane == 0) {
+        // Q K^T is issued 128 keys wide (8 instructions per tile and group, 64 cycles each on the tensor
+        // core): narrower instructions cost nearly as much to issue.
+        {
             bool ok = true;
             int gt = 0;               // KV tiles before this item (all items): ring position
             int cnt0 = 0, cnt1 = 0;   // tiles whose P V has been issued, per group: phase of the P hand-off
@@ -426,29 +469,46 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             TItem it_next = load_titem(head_work, i0 < i1);
             const long long t_loop = trace_clock();
             long long tr_p = 0, tr_kv = 0, tr_item = 0, tr_qk = 0, tr_pv = 0;      // time-stamp build: cycles waiting for P, for K/V, for an item's Q and O
+            int ev = 0;                                                            // time-stamp build: event log position
             for (int ii = i0; ii < i1 && ok; ++ii, ++item_no) {
                 const TItem it = it_next;
                 it_next = load_titem(p.works + ii + 1, ii + 1 < i1);      // in flight while this item runs
                 const int ntiles = (it.kv_end - it.kv0 + kTile - 1) / kTile;
                 const bool dual = it.ntok * G > kTile;
                 const long long t_item = trace_clock();
+                if (lane == 0) trace_event(0, ev, 1);
                 ok = mbar_wait_spin(bar(kQFull), (uint32_t)item_no & 1u, abort_flag, p.status, 22);
                 // S and O of the previous item are in use until its epilogue is over
                 if (ok && item_no > 0) ok = mbar_wait_spin(bar(kOFree), (uint32_t)(item_no - 1) & 1u, abort_flag, p.status, 27);
                 tr_item += trace_clock() - t_item;
+                if (lane == 0) trace_event(0, ev, 2);
                 if (ok) tc_fence_after();
                 auto tile_pages = [&](int j) { return (min(kTile, it.kv_end - (it.kv0 + j * kTile)) + kPage - 1) / kPage; };
+                // Hand-offs the MMAs of a turn wait for.  K/V tiles first (they are normally there already),
+                // P last, so that nothing stands between its arrival and the first MMA.
+                auto wait_k = [&](int j) {
+                    const int pos = ring_pos_k(gt + j), s = pos % kRing;
+                    const long long tw = trace_clock();
+                    ok = ok && mbar_wait_spin(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
+                    tr_kv += trace_clock() - tw;
+                };
+                auto wait_v = [&](int j) {
+                    const int pos = ring_pos_v(gt + j), s = pos % kRing;
+                    const long long tw = trace_clock();
+                    ok = ok && mbar_wait_spin(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
+                    tr_kv += trace_clock() - tw;
+                };
+                auto wait_p = [&](int b) {
+                    const long long tw = trace_clock();
+                    ok = ok && mbar_wait_spin(bar(kPFull0 + 2 * b), (uint32_t)(b ? cnt1 : cnt0) & 1u, abort_flag, p.status, 26);
+                    tr_p += trace_clock() - tw;
+                };
                 // S[b] <- Q[qt] K_j^T, then one commit: it tells group b that S[b] is complete and, because MMAs
                 // complete in issue order, that every MMA in front of it is done as well (the group releases
                 // the ring slots on that knowledge: a second commit per batch costs the tensor pipe ~90 cycles)
-                auto issue_qk = [&](int j, int b) {
-                    const int pos = ring_pos_k(gt + j), s = pos % kRing;
-                    const long long tw = trace_clock();
-                    ok = mbar_wait_spin(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 21);
+                auto emit_qk = [&](int j, int b) {
                     const long long ti = trace_clock();
-                    tr_kv += ti - tw;
-                    if (!ok) return;
-                    tc_fence_after();
+                    const int s = ring_pos_k(gt + j) % kRing;
                     const uint32_t idesc = instr_desc(16u * (uint32_t)tile_pages(j), 0);
                     const uint32_t d = tmem + kColS + 128u * (uint32_t)b;
                     const uint64_t qd = smem_desc(sbase + kOffQ + (dual ? (uint32_t)b * kTileBytes : 0u), 16, 1024);
@@ -457,62 +517,77 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     for (int ks = 0; ks < kD / 16; ++ks) {
                         // the address field counts 16-byte units and cannot carry out of its 14 bits here
                         const uint64_t off = (uint64_t)(((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4);
-                        mma_f16(d, qd + off, kd + off, idesc, ks > 0);
+                        if (elect_one()) mma_f16(d, qd + off, kd + off, idesc, ks > 0);
                     }
-                    mma_commit(bar(kSFull0 + 2 * b));
+                    if (elect_one()) mma_commit(bar(kSFull0 + 2 * b));
                     tr_qk += trace_clock() - ti;
+                    if (lane == 0) trace_event(0, ev, 14 + b);
                 };
                 // O[b] (+)= P[b] V_j with P[b] in tensor memory; fresh: first P V of the item into O[b];
                 // last: the group's last tile of the item, the only one whose completion is signalled by itself
-                auto issue_pv = [&](int j, int b, bool fresh, bool last) {
-                    const int pos = ring_pos_v(gt + j), s = pos % kRing;
-                    const long long tw = trace_clock();
-                    ok = mbar_wait_spin(bar(kPFull0 + 2 * b), (uint32_t)(b ? cnt1 : cnt0) & 1u, abort_flag, p.status, 26);
-                    const long long tv = trace_clock();
-                    tr_p += tv - tw;
-                    ok = ok && mbar_wait_spin(bar(kRingFull0 + s), (uint32_t)(pos / kRing) & 1u, abort_flag, p.status, 24);
+                auto emit_pv = [&](int j, int b, bool fresh, bool last) {
                     const long long ti = trace_clock();
-                    tr_kv += ti - tv;
-                    if (!ok) return;
-                    tc_fence_after();
+                    const int s = ring_pos_v(gt + j) % kRing;
                     const int npg = tile_pages(j);
                     const uint32_t pcol = tmem + kColS + 128u * (uint32_t)b;
                     const uint64_t vd = smem_desc(sbase + kOffRing + s * kTileBytes, kHalfBytes, 1024);
-                    for (int ks = 0; ks < npg; ++ks)
-                        mma_f16_ta(tmem + kColO + 128u * (uint32_t)b, pcol + 8u * (uint32_t)ks, vd + (uint64_t)(ks * 128),
-                                   idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
-                    if (last) mma_commit(bar(kPvDone0 + 2 * b));
+                    const uint32_t ocol = tmem + kColO + 128u * (uint32_t)b;
+                    if (npg == kTile / kPage) {
+#pragma unroll
+                        for (int ks = 0; ks < kTile / kPage; ++ks)
+                            if (elect_one()) mma_f16_ta(ocol, pcol + 8u * (uint32_t)ks, vd + (uint64_t)(ks * 128), idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
+                    } else {
+                        for (int ks = 0; ks < npg; ++ks)
+                            if (elect_one()) mma_f16_ta(ocol, pcol + 8u * (uint32_t)ks, vd + (uint64_t)(ks * 128), idesc_pv, (!fresh || ks > 0) ? 1u : 0u);
+                    }
+                    if (last && elect_one()) mma_commit(bar(kPvDone0 + 2 * b));
                     if (b) ++cnt1; else ++cnt0;
                     tr_pv += trace_clock() - ti;
+                    if (lane == 0) trace_event(0, ev, 26 + b);
+                };
+                auto first_qk = [&](int j, int b) {
+                    wait_k(j);
+                    if (!ok) return;
+                    tc_fence_after();
+                    emit_qk(j, b);
+                };
+                // One turn of group b: the P V of its tile j and at once the Q K^T of its next tile jn (-1: none),
+                // sixteen MMAs issued back to back once everything they read is there.
+                auto turn = [&](int j, int b, bool fresh, int jn) {
+                    if (lane == 0) trace_event(0, ev, 20 + b);
+                    wait_v(j);
+                    if (jn >= 0) wait_k(jn);
+                    wait_p(b);
+                    if (lane == 0) trace_event(0, ev, 22 + b);
+                    if (!ok) return;
+                    tc_fence_after();
+                    emit_pv(j, b, fresh, jn < 0);
+                    if (jn >= 0) emit_qk(jn, b);
                 };
                 if (dual) {
                     // both groups on every tile: group b owns row tile b
-                    if (ok) issue_qk(0, 0);
-                    if (ok) issue_qk(0, 1);
+                    first_qk(0, 0);
+                    if (ok) first_qk(0, 1);
                     for (int j = 0; j < ntiles && ok; ++j)
-                        for (int b = 0; b < 2 && ok; ++b) {
-                            issue_pv(j, b, j == 0, j + 1 == ntiles);
-                            if (ok && j + 1 < ntiles) issue_qk(j + 1, b);
-                        }
+                        for (int b = 0; b < 2 && ok; ++b) turn(j, b, j == 0, j + 1 < ntiles ? j + 1 : -1);
                 } else {
                     // one row tile: the groups take alternate KV tiles
-                    if (ok) issue_qk(0, 0);
-                    if (ok && ntiles > 1) issue_qk(1, 1);
-                    for (int j = 0; j < ntiles && ok; ++j) {
-                        issue_pv(j, j & 1, j < 2, j + 2 >= ntiles);
-                        if (ok && j + 2 < ntiles) issue_qk(j + 2, j & 1);
-                    }
+                    first_qk(0, 0);
+                    if (ok && ntiles > 1) first_qk(1, 1);
+                    for (int j = 0; j < ntiles && ok; ++j) turn(j, j & 1, j < 2, j + 2 < ntiles ? j + 2 : -1);
                 }
                 gt += ntiles;
             }
-            trace_set(8, tr_p);
-            trace_set(9, tr_kv);
-            trace_set(10, trace_clock() - t_loop);
-            trace_set(14, tr_item);
-            trace_set(2, tr_qk);
-            trace_set(3, tr_pv);
+            if (lane == 0) {
+                trace_set(8, tr_p);
+                trace_set(9, tr_kv);
+                trace_set(10, trace_clock() - t_loop);
+                trace_set(14, tr_item);
+                trace_set(2, tr_qk);
+                trace_set(3, tr_pv);
+            }
             // make sure nothing is still running on the tensor core before tensor memory is released
-            mma_commit(bar(kMmaDrain));
+            if (elect_one()) mma_commit(bar(kMmaDrain));
             const long long t0 = clock64();
             while (!mbar_try_wait(bar(kMmaDrain), 0) && clock64() - t0 < kWaitCycles) {}
         }
@@ -533,6 +608,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
         int item_no = 0;
         bool ok = true;
         long long tr_wait = 0, tr_work = 0, tr_tiles = 0;      // time-stamp build: cycles waiting for S, cycles from S to P, tiles
+        int ev = 0;                                            // time-stamp build: event log position (lane 0 of each warp)
         // This thread's share of an item's Q.  Dual items: the whole row 128 b + m (16 chunks of 16
         // bytes) into Q[b]; otherwise value half b of row m (8 chunks) into Q[0].  The next item's Q is
         // fetched at the end of the current item's KV loop, ahead of the epilogue.
@@ -576,6 +652,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             }
             fence_async_smem();
             mbar_arrive(bar(kQFull));
+            if (lane == 0) trace_event(1 + warp, ev, 37);
             it_next = load_titem(p.works + ii + 1, ii + 1 < i1);
             const int lim_row = row_valid ? min(it.kv_limit0 + t, it.kv_end) : 0;   // keys [0, lim_row) visible
             float m_ref = -INFINITY;                     // reference maximum (log2 domain)
@@ -586,8 +663,10 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 // S[b] complete; it was issued after the P V of this group's previous tile finished, so
                 // O[b] is at rest as well
                 const long long tw = trace_clock();
-                ok = mbar_wait_warp(bar(kSFull0 + 2 * b), (uint32_t)(cnt + mine) & 1u, abort_flag, p.status, 31);
+                if (lane == 0) trace_event(1 + warp, ev, 30);
+                ok = __all_sync(0xffffffffu, mbar_wait_spin(bar(kSFull0 + 2 * b), (uint32_t)(cnt + mine) & 1u, abort_flag, p.status, 31));
                 const long long ts = trace_clock();
+                if (lane == 0) trace_event(1 + warp, ev, 31);
                 tr_wait += ts - tw;
                 ++tr_tiles;
                 if (!ok) break;
@@ -691,12 +770,15 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 }
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(kPFull0 + 2 * b));
+                __syncwarp();      // 128 arrivals on one barrier word would take turns; the warp's lanes are ordered here instead
+                if (lane == 0) mbar_arrive(bar(kPFull0 + 2 * b));
                 tr_work += trace_clock() - ts;
+                if (lane == 0) trace_event(1 + warp, ev, 32);
             }
             if (!ok) break;
             const float l_sum = (l2.x + l2.y) + (l2b.x + l2b.y);
             load_q(it_next, q_next);        // in flight during the epilogue
+            if (lane == 0) trace_event(1 + warp, ev, 33);
             // ---- epilogue.  The groups' (max, sum) go through columns 0-1 of their S buffers, which are
             // idle from the group's last P V until the next item's first Q K^T.
             if (mine > 0) {
@@ -704,6 +786,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                 if (!ok) break;
                 ++pv_cnt;
                 tc_fence_after();
+                if (lane == 0) trace_event(1 + warp, ev, 34);
                 // the V tile of the group's last tile goes back to the producers
                 if (m == 0 && (!dual || b == 1))
                     mbar_arrive(bar(kRingEmpty0 + ring_pos_v(gt + (dual ? ntiles - 1 : b + 2 * (mine - 1))) % kRing));
@@ -715,6 +798,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             ok = mbar_wait_warp(bar(kStats), (uint32_t)item_no & 1u, abort_flag, p.status, 35);
             if (!ok) break;
             tc_fence_after();
+            if (lane == 0) trace_event(1 + warp, ev, 35);
             const size_t hq = (size_t)it.kv_head * G + g;
             const size_t prow = it.partial_row0 < 0 ? 0 : (size_t)it.partial_row0 + t;
             float w0, w1, lse2;          // weights of O[0] and O[1] in this thread's output row
@@ -817,6 +901,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
             }
             tc_fence_before();
             mbar_arrive(bar(kOFree));
+            if (lane == 0) trace_event(1 + warp, ev, 36);
             cnt += mine;
             gt += ntiles;
         }

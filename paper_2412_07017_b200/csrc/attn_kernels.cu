@@ -258,4 +258,11 @@ cudaError_t launch_attention(const DevPlan& p, const void* q, const void* kv_poo
 extern "C" int asynclm_trace_read(unsigned long long* out) {
     return cudaMemcpyFromSymbol(out, asynclm::g_trace, sizeof(asynclm::g_trace)) == cudaSuccess ? 0 : -5;
 }
+// The event log of the first CTAs: out [4][11][512] unsigned 64-bit (cycle << 8 | event); clears it.
+extern "C" int asynclm_trace_events_read(unsigned long long* out) {
+    if (cudaMemcpyFromSymbol(out, asynclm::g_events, sizeof(asynclm::g_events)) != cudaSuccess) return -5;
+    void* dev = nullptr;
+    if (cudaGetSymbolAddress(&dev, asynclm::g_events) != cudaSuccess) return -5;
+    return cudaMemset(dev, 0, sizeof(asynclm::g_events)) == cudaSuccess ? 0 : -5;
+}
 #endif

@@ -75,7 +75,16 @@ __device__ __forceinline__ void trace_set(int slot, unsigned long long v) {
     if (blockIdx.x < kTraceCtas) g_trace[blockIdx.x][slot] = v;
 }
 __device__ __forceinline__ long long trace_clock() { return clock64(); }
+// Event log of the first kEventCtas CTAs: (SM cycle counter << 8 | event id) in the order a role
+// (one thread) records them; `n` is the role's own count.
+constexpr int kEventCtas = 4, kEventRoles = 11, kEventsPerRole = 512;
+static __device__ unsigned long long g_events[kEventCtas][kEventRoles][kEventsPerRole];
+__device__ __forceinline__ void trace_event(int role, int& n, int id) {
+    if (blockIdx.x < kEventCtas && n < kEventsPerRole)
+        g_events[blockIdx.x][role][n++] = ((unsigned long long)clock64() << 8) | (unsigned)id;
+}
 #else
+__device__ __forceinline__ void trace_event(int, int&, int) {}
 __device__ __forceinline__ long long trace_clock() { return 0; }
 __device__ __forceinline__ void trace_mark(int) {}
 __device__ __forceinline__ void trace_add(int, unsigned long long) {}
