@@ -255,8 +255,13 @@ int asynclm_step(const asynclm_plan_t* plan, const void* q, const void* k_new, c
 
 /*
  * Reads the device status word of the plan's workspace (synchronises `stream`).  *host_out is 0
- * if no kernel reported a problem, otherwise a code naming the bounded wait that ran out.  Returns
- * ASYNCLM_OK or ASYNCLM_ERR_DEVICE_STATUS / ASYNCLM_ERR_CUDA.
+ * if no kernel reported a problem, otherwise a code naming the bounded wait that ran out (1-39).
+ * A library built with -DASYNCLM_DEBUG (build.py --debug) also checks, on the device, every page id
+ * it is about to turn into an address and reports the first bad one here instead of using it:
+ * 41 the append's row slot, 42 a span tile's page, 43 a decode chunk's page, 44 the append inside
+ * asynclm_step; the access is left out (span tiles get zeros, decode chunks read page 0), nothing
+ * faults.  The ordinary build relies on asynclm_plan, which validates every id on the host.
+ * Returns ASYNCLM_OK or ASYNCLM_ERR_DEVICE_STATUS / ASYNCLM_ERR_CUDA.
  */
 int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out);
 

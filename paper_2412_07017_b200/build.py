@@ -14,6 +14,9 @@ LIB = os.path.join(CSRC, "libasynclm.so")
 # A second build with per-CTA time stamps compiled in (-DASYNCLM_TRACE, asynclm_trace_read): for
 # performance work only; the binding loads it when ASYNCLM_LIBRARY points at it.
 TRACE_LIB = os.path.join(CSRC, "libasynclm_trace.so")
+# A third build with device-side checks of every page id a kernel turns into an address (-DASYNCLM_DEBUG):
+# a bad id sets the plan's status word and the access is left out.  For bringing up a new caller.
+DEBUG_LIB = os.path.join(CSRC, "libasynclm_debug.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -42,16 +45,16 @@ def find_nvcc():
     return nvcc if os.path.exists(nvcc) else None
 
 
-def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
-    lib = TRACE_LIB if trace else LIB
-    if not force and not trace and not is_stale():
+def build(force: bool = False, verbose: bool = False, trace: bool = False, debug: bool = False) -> str:
+    lib = TRACE_LIB if trace else DEBUG_LIB if debug else LIB
+    if not force and not trace and not debug and not is_stale():
         return lib
     nvcc = find_nvcc()
     if nvcc is None:
         raise RuntimeError("nvcc not found; cannot build libasynclm.so")
     tmp = lib + f".tmp{os.getpid()}"
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-        (["-DASYNCLM_TRACE"] if trace else []) + ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
+        (["-DASYNCLM_TRACE"] if trace else []) + (["-DASYNCLM_DEBUG"] if debug else []) + ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + sources()
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + proc.stdout + proc.stderr)
@@ -62,4 +65,4 @@ def build(force: bool = False, verbose: bool = False, trace: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, trace="--trace" in sys.argv, debug="--debug" in sys.argv))

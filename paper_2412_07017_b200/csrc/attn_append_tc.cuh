@@ -408,7 +408,9 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                     const int c = lane & 15;
                     const uint32_t dst_half = ring + s * kTileBytes + (uint32_t)(c >> 3) * kHalfBytes;
                     for (int pg = 0; pg < npages; ++pg) {
-                        const int64_t page = __shfl_sync(0xffffffffu, pages_cur, (t - t0) * kPagesPerTile + pg);
+                        int64_t page = __shfl_sync(0xffffffffu, pages_cur, (t - t0) * kPagesPerTile + pg);
+                        const bool page_good = page_ok(page, p.num_pages, p.status, kStatusBadPageSpan);      // checked build only
+                        if (!page_good) page = 0;      // the tile gets zeros in its place
                         const uint8_t* src_page = reinterpret_cast<const uint8_t*>(
                             pool + pool_row_offset(page, which, cur.kv_head, 0, Hkv, kD));
 #pragma unroll
@@ -416,7 +418,7 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                             const int slot = rr * 2 + (lane >> 4);
                             const int row = pg * kPage + slot;
                             cp_async16(dst_half + (uint32_t)row * 128u + (uint32_t)(((c & 7) ^ (row & 7)) << 4),
-                                       src_page + slot * (kD * 2) + c * 16, row < rows ? 16u : 0u);
+                                       src_page + slot * (kD * 2) + c * 16, (row < rows && page_good) ? 16u : 0u);
                         }
                     }
                     cp_async_arrive(bar(kRingFull0 + s));

@@ -505,8 +505,10 @@ __device__ __forceinline__ void decode_body(const DevPlan& p, const CUtensorMap*
                                               (uint32_t)(npages * Geo::PAGE_BYTES + (first ? cur.ntok * G * D * 2 : 0)));
                     }
                     __syncwarp();
-                    const int page = __shfl_sync(0xffffffffu, pages_cur,
-                                                 (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
+                    int page = __shfl_sync(0xffffffffu, pages_cur,
+                                           (t - t0) * kPagesPerTile + (lane < kPagesPerTile ? lane : 0));
+                    // checked build only: a bad id is replaced by page 0 (the copy must happen: the stage counts its bytes)
+                    if (lane < npages && !page_ok(page, p.num_pages, p.status, kStatusBadPageWarp)) page = 0;
                     if (lane == 0) { if (n == 0) trace_mark(2); trace_add(6, 1); if (first) trace_add(5, 1); }
                     if (lane < npages)
                         tma_page_kv(smem_u32(stage_base + (size_t)s * Geo::STAGE_BYTES + (size_t)lane * Geo::PAGE_BYTES),

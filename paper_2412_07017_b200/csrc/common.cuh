@@ -91,6 +91,21 @@ __device__ __forceinline__ void trace_add(int, unsigned long long) {}
 __device__ __forceinline__ void trace_set(int, unsigned long long) {}
 #endif
 
+// Checked build (-DASYNCLM_DEBUG, see build.py): every page id a kernel is about to turn into an address is
+// compared with the pool's size first; a bad one puts `code` into the status word (the first one wins)
+// and the caller leaves the access out.  The ordinary build relies on the planner, which validates every
+// id on the host, and compiles the check away.
+#ifdef ASYNCLM_DEBUG
+__device__ __forceinline__ bool page_ok(int64_t page, int64_t num_pages, int32_t* status, int code) {
+    if (page >= 0 && page < num_pages) return true;
+    atomicCAS(status, 0, code);
+    return false;
+}
+#else
+__device__ __forceinline__ bool page_ok(int64_t, int64_t, int32_t*, int) { return true; }
+#endif
+constexpr int kStatusBadPageAppend = 41, kStatusBadPageSpan = 42, kStatusBadPageWarp = 43, kStatusBadPageStep = 44;
+
 // Element offset of the first value of (page, K|V, kv head, slot) in the pool.
 __device__ __forceinline__ size_t pool_row_offset(int64_t page, int which, int kv_head, int slot,
                                                   int num_kv_heads, int head_dim) {
@@ -117,20 +132,23 @@ __device__ __forceinline__ void append_rows_of_item(const DevPlan& p, const Appe
     for (int base = lane; base < total; base += 32 * kBatch) {
         uint4 val[kBatch];
         size_t dst[kBatch];
+        bool ok[kBatch];
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
             const int i = base + 32 * j;
             if (i < total) {
                 const int pos = lo + i / (2 * vpr), r = i % (2 * vpr);
                 const int which = r / vpr, vec = r % vpr;
-                const int64_t page = __ldg(p.page_indices + w.page0 + (pos - w.kv0) / kPage);
+                int64_t page = __ldg(p.page_indices + w.page0 + (pos - w.kv0) / kPage);
+                ok[j] = page_ok(page, p.num_pages, p.status, kStatusBadPageStep);
+                if (!ok[j]) page = 0;
                 val[j] = ldg_nc_v4((which ? v_new : k_new) + ((size_t)(w.q_seq0 + pos - ctx) * p.num_kv_heads + w.kv_head) * vpr + vec);
                 dst[j] = pool_row_offset(page, which, w.kv_head, pos % kPage, p.num_kv_heads, p.head_dim) / 8 + vec;
             }
         }
 #pragma unroll
         for (int j = 0; j < kBatch; ++j)
-            if (base + 32 * j < total) pool[dst[j]] = val[j];
+            if (base + 32 * j < total && ok[j]) pool[dst[j]] = val[j];
     }
 }
 

@@ -28,6 +28,7 @@ kv_append_kernel(DevPlan p, const uint4* __restrict__ k_new, const uint4* __rest
         // the slot and the source row are fetched side by side instead of through four dependent loads
         const int64_t ps = __ldg(p.row_slot + r);
         const uint4 val = ldg_nc_v4((which ? v_new : k_new) + ((size_t)r * p.num_kv_heads + h) * vpr + vec);
+        if (!page_ok(ps / kPage, p.num_pages, p.status, kStatusBadPageAppend)) continue;
         const size_t dst = pool_row_offset(ps / kPage, which, h, (int)(ps % kPage), p.num_kv_heads, p.head_dim) / 8 + vec;
         pool[dst] = val;
     }

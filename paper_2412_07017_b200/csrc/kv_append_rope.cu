@@ -67,6 +67,7 @@ kv_append_rope_kernel(DevPlan p, const uint4* __restrict__ k_new, const uint4* _
         }
         if (is_k) {
             const int64_t ps = __ldg(p.row_slot + r);
+            if (!page_ok(ps / kPage, p.num_pages, p.status, kStatusBadPageAppend)) continue;
             const size_t dst = pool_row_offset(ps / kPage, 0, h, (int)(ps % kPage), heads_k, d) / 8;
             pool[dst + v] = olo;
             pool[dst + v + half_vecs] = ohi;

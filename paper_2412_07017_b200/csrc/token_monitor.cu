@@ -269,11 +269,13 @@ extern "C" int asynclm_token_monitor_step(const void* logits, int32_t dtype, int
         ((uintptr_t)workspace & 15) != 0 || ((size_t)row_stride * esz) % 16 != 0 || batch > 65535)
         return ASYNCLM_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
-    // slices per row: enough CTAs of 32 KB in flight to fill the machine several times over, at least
-    // one pass of kMonVecs vectors per thread each
+    // slices per row: about two CTAs per SM in all, at least one pass of kMonVecs vectors per thread each.
+    // Fewer, longer CTAs measure faster than many short ones (256 rows of 128 256 bf16: 20.5 us with one
+    // or two slices per row, 22.6 with three or four, 24.7 with five to seven): every CTA ends on a
+    // block-wide reduction, an atomic and a fence.
     const int nvec = vocab / (16 / (int)esz);
     const int max_slices = std::max(1, nvec / (kMonThreads * kMonVecs));
-    const int slices = std::max(1, std::min(max_slices, (148 * 16 + batch - 1) / batch));
+    const int slices = std::max(1, std::min(max_slices, (148 * 2 + batch - 1) / batch));
     const dim3 grid((unsigned)slices, (unsigned)batch);
     if (dtype == ASYNCLM_DTYPE_BF16)
         token_monitor_kernel<__nv_bfloat16><<<grid, kMonThreads, 0, s>>>((const __nv_bfloat16*)logits, vocab, row_stride, *tokens,
