@@ -99,6 +99,21 @@ extern "C" int asynclm_step(const asynclm_plan_t* plan, const void* q, const voi
     return cuda_status(launch_lse_merge(plan->dev, out, lse, s));
 }
 
+#ifdef ASYNCLM_DEBUG
+// Checked build only (not part of the public header): the span body's K producer of CTA 0 will not hand
+// over its tile-th K tile (1-based; 0 switches it off) in the launches that follow.  The waits that depend
+// on that tile (the MMA warp's for the tile, a softmax group's for its scores, the producers' for a free
+// slot) then run out after their cycle budget (about a second); the first to do so records its code
+// (11, 12, 21, 24, 26 or 31), every role of the CTA leaves through the common exit, tensor memory is
+// released and asynclm_last_device_status reports the code.  The GPU neither faults nor hangs: this is
+// the test of the bounded waits.  The CTA's output rows are undefined in such a launch.
+extern "C" int asynclm_debug_stall_span_tile(asynclm_plan_t* plan, int32_t tile) {
+    if (!plan || plan->magic != asynclm::kPlanMagic || tile < 0) return ASYNCLM_ERR_INVALID_ARG;
+    plan->dev.debug_stall_tile = tile;
+    return ASYNCLM_OK;
+}
+#endif
+
 extern "C" int asynclm_last_device_status(const asynclm_plan_t* plan, void* stream, int32_t* host_out) {
     if (!runnable(plan) || !host_out) return ASYNCLM_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;

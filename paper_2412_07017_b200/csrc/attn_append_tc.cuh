@@ -421,6 +421,10 @@ __device__ __forceinline__ void tc_body(const DevPlan& p, const __nv_bfloat16* _
                                        src_page + slot * (kD * 2) + c * 16, (row < rows && page_good) ? 16u : 0u);
                         }
                     }
+#ifdef ASYNCLM_DEBUG
+                    // checked build: a test may ask for one hand-off to be left out, to see a bounded wait run out
+                    if (!(which == 0 && blockIdx.x == 0 && p.debug_stall_tile == n + 1))
+#endif
                     cp_async_arrive(bar(kRingFull0 + s));
                     if (lane == 0) trace_event(9 + which, ev, 44);
                     // page ids of the next group of tiles (or of the next item), requested only after this

@@ -97,6 +97,8 @@ struct DevPlan {
     int32_t num_q_heads, num_kv_heads, head_dim, group;
     int64_t num_pages;
     float sm_scale;
+    int32_t debug_stall_tile;        // checked build only, 0 = off: the K producer of CTA 0 leaves out the hand-off
+                                     // of its n-th span tile, so that the wait for it runs out (see api.cu)
 };
 
 }  // namespace asynclm

@@ -77,5 +77,43 @@ def main():
     print(json.dumps(result))
 
 
+def wait_expiry():
+    """A hand-off that never comes: the bounded waits run out, the status word names one of them, the
+    context stays usable and the next step is correct."""
+    import ctypes
+    torch.cuda.set_device(0)
+    shape = W.Shape(32, 8, 128, 16)
+    wl = W.make_single_step("stall", shape, [1500, 1200], [64, 64], seed=78)      # spans only: the span kernel alone
+    st = wl.steps[0]
+    pool = to_dev(wl.kv_pool)
+    q, kn, vn = to_dev(st.q), to_dev(st.k_new), to_dev(st.v_new)
+    _, ref_out, ref_lse = oracle_step(wl, st)
+    lib = B.load()
+    lib.asynclm_debug_stall_span_tile.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+    lib.asynclm_debug_stall_span_tile.restype = ctypes.c_int
+
+    def run(stall):
+        out = torch.zeros((st.total_q, shape.num_q_heads, shape.head_dim), dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros((st.total_q, shape.num_q_heads), dtype=torch.float32, device="cuda")
+        plan = B.asynclm_plan(shape, wl.num_pages, st.q_indptr, st.kv_len_before, st.page_indptr, st.page_indices)
+        assert plan.info["num_items_tensor"] == plan.info["num_items"] > 0
+        assert lib.asynclm_debug_stall_span_tile(ctypes.c_void_p(plan.handle), stall) == 0
+        B.asynclm_kv_append(plan, kn, vn, pool)
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        B.asynclm_attn_mixed(plan, q, pool, out, lse)
+        t1.record()
+        torch.cuda.synchronize()
+        return B.last_device_status(plan), to_bits(out), lse.cpu().numpy(), t0.elapsed_time(t1)
+
+    status, _, _, ms = run(2)
+    res = {"stalled_status": status, "stalled_ms": ms}
+    status, out, lse, ms = run(0)
+    assert_close(out, lse, ref_out, ref_lse, what="the step after a wait ran out")
+    res.update({"next_status": status, "next_ms": ms})
+    print(json.dumps(res))
+
+
 if __name__ == "__main__":
-    main()
+    wait_expiry() if sys.argv[1:] == ["wait"] else main()
