@@ -20,7 +20,7 @@ DEBUG_LIB = os.path.join(CSRC, "libasynclm_debug.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math", "-Xcompiler", "-fPIC", "-shared",
+    "--use_fast_math", "-Xcompiler", "-fPIC", "-shared", "--threads", "0",
 ]
 
 
